@@ -1,0 +1,184 @@
+"""ctypes front end of the fp64 CPU oracle.  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package; the CUDA library and its binding never do.  The arithmetic lives
+in ``rstitch_oracle.c`` (plain C, fp64); this file only builds it with gcc,
+marshals numpy arrays and returns numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rstitch_oracle.c")
+_LIB = os.path.join(_HERE, "librstitch_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+                               "-ffp-contract=off", "-fno-fast-math", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        c = ctypes
+        u16p, i32p, f64p, u8p = (c.POINTER(c.c_uint16), c.POINTER(c.c_int32),
+                                 c.POINTER(c.c_double), c.POINTER(c.c_uint8))
+        lib.oracle_num_threads.restype = c.c_int
+        lib.oracle_logits_row.argtypes = [u16p, u16p, c.c_int, c.c_int, f64p]
+        lib.oracle_logits_row.restype = None
+        lib.oracle_greedy.argtypes = [f64p, c.c_int, i32p, f64p]
+        lib.oracle_greedy.restype = None
+        lib.oracle_entropy_nats.argtypes = [f64p, c.c_int]
+        lib.oracle_entropy_nats.restype = c.c_double
+        lib.oracle_entropy_normalized.argtypes = [f64p, c.c_int]
+        lib.oracle_entropy_normalized.restype = c.c_double
+        lib.oracle_rule.argtypes = [c.c_double, c.c_double]
+        lib.oracle_rule.restype = c.c_uint8
+        lib.oracle_head_rows.argtypes = [u16p, i32p, u16p, c.c_int, c.c_int, c.c_int,
+                                         i32p, f64p, f64p, f64p]
+        lib.oracle_head_rows.restype = None
+        lib.oracle_mask.argtypes = [f64p, i32p, c.c_int, c.c_int, c.c_double, u8p]
+        lib.oracle_mask.restype = None
+        lib.oracle_compact.argtypes = [u8p, c.c_int, i32p, i32p]
+        lib.oracle_compact.restype = None
+        lib.oracle_spans.argtypes = [i32p, c.c_int32, i32p, i32p, i32p, i32p]
+        lib.oracle_spans.restype = None
+        _lib = lib
+    return _lib
+
+
+def _p(a: Optional[np.ndarray], ct):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def _u16(a):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, "bf16 inputs are passed as uint16 bit patterns"
+    return a
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def logits_row(hidden_row: np.ndarray, w_head: np.ndarray) -> np.ndarray:
+    """z[v] = sum_k hidden[k] * W_head[v, k] in fp64 (Section 3.1)."""
+    h, w = _u16(hidden_row), _u16(w_head)
+    V, d = w.shape
+    assert h.shape == (d,)
+    z = np.empty(V, dtype=np.float64)
+    _load().oracle_logits_row(_p(h, ctypes.c_uint16), _p(w, ctypes.c_uint16), d, V,
+                              _p(z, ctypes.c_double))
+    return z
+
+
+def greedy(z: np.ndarray):
+    """(token, top-2 gap): lowest index of the maximum logit."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    tok, gap = ctypes.c_int32(0), ctypes.c_double(0.0)
+    _load().oracle_greedy(_p(z, ctypes.c_double), z.size, ctypes.byref(tok), ctypes.byref(gap))
+    return int(tok.value), float(gap.value)
+
+
+def entropy_nats(z: np.ndarray) -> float:
+    """Softmax entropy of a logit vector, nats (numerator of Eq. 1)."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    return float(_load().oracle_entropy_nats(_p(z, ctypes.c_double), z.size))
+
+
+def entropy_normalized(z: np.ndarray) -> float:
+    """Eq. 1: entropy / log V."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    return float(_load().oracle_entropy_normalized(_p(z, ctypes.c_double), z.size))
+
+
+def rule(H: float, tau: float) -> int:
+    """Eq. 2 / Algorithm 1: 1 iff H > tau (NaN routes to the LLM)."""
+    return int(_load().oracle_rule(float(H), float(tau)))
+
+
+def head_rows(hidden: np.ndarray, w_head: np.ndarray, row_idx: Optional[np.ndarray] = None):
+    """Per-row (tok int32, H nats, H / log V, top-2 gap) for R rows."""
+    h, w = _u16(hidden), _u16(w_head)
+    V, d = w.shape
+    assert h.ndim == 2 and h.shape[1] == d
+    if row_idx is not None:
+        row_idx = np.ascontiguousarray(row_idx, dtype=np.int32)
+        R = row_idx.size
+        assert R == 0 or (row_idx.min() >= 0 and row_idx.max() < h.shape[0])
+    else:
+        R = h.shape[0]
+    tok = np.zeros(R, dtype=np.int32)
+    H = np.zeros(R, dtype=np.float64)
+    Hn = np.zeros(R, dtype=np.float64)
+    gap = np.zeros(R, dtype=np.float64)
+    if R:
+        _load().oracle_head_rows(_p(h, ctypes.c_uint16), _p(row_idx, ctypes.c_int32),
+                                 _p(w, ctypes.c_uint16), R, d, V, _p(tok, ctypes.c_int32),
+                                 _p(H, ctypes.c_double), _p(Hn, ctypes.c_double),
+                                 _p(gap, ctypes.c_double))
+    return tok, H, Hn, gap
+
+
+def mask(H_nats: np.ndarray, tau: float, B: Optional[int] = None,
+         row_seq: Optional[np.ndarray] = None) -> np.ndarray:
+    """Per-sequence route mask (uint8 [B]); decision row = last row of each span."""
+    H = np.ascontiguousarray(H_nats, dtype=np.float64)
+    R = H.size
+    if B is None:
+        B = R
+    if row_seq is not None:
+        row_seq = np.ascontiguousarray(row_seq, dtype=np.int32)
+        assert row_seq.size == R
+    out = np.zeros(B, dtype=np.uint8)
+    _load().oracle_mask(_p(H, ctypes.c_double), _p(row_seq, ctypes.c_int32), R, B, float(tau),
+                        _p(out, ctypes.c_uint8))
+    return out
+
+
+def compact(mask_u8: np.ndarray):
+    """(llm_idx int32 [count], count): ascending indices of the routed sequences."""
+    m = np.ascontiguousarray(mask_u8, dtype=np.uint8)
+    idx = np.zeros(max(m.size, 1), dtype=np.int32)
+    cnt = ctypes.c_int32(0)
+    _load().oracle_compact(_p(m, ctypes.c_uint8), m.size, _p(idx, ctypes.c_int32), ctypes.byref(cnt))
+    return idx[:cnt.value].copy(), int(cnt.value)
+
+
+def spans(llm_idx: np.ndarray, seq_len: np.ndarray, kv_len: np.ndarray):
+    """(llm_span [count], llm_row_off [count + 1]) of the routed sequences."""
+    idx = np.ascontiguousarray(llm_idx, dtype=np.int32)
+    sl = np.ascontiguousarray(seq_len, dtype=np.int32)
+    kl = np.ascontiguousarray(kv_len, dtype=np.int32)
+    n = idx.size
+    span = np.zeros(max(n, 1), dtype=np.int32)
+    off = np.zeros(n + 1, dtype=np.int32)
+    _load().oracle_spans(_p(idx, ctypes.c_int32), n, _p(sl, ctypes.c_int32), _p(kl, ctypes.c_int32),
+                         _p(span, ctypes.c_int32), _p(off, ctypes.c_int32))
+    return span[:n].copy(), off
+
+
+def route(hidden, w_head, tau_nats, row_idx=None, row_seq=None, B=None, seq_len=None, kv_len=None):
+    """The whole decision of one step, as a dict of numpy arrays."""
+    tok, H, Hn, gap = head_rows(hidden, w_head, row_idx)
+    m = mask(H, tau_nats, B=B, row_seq=row_seq)
+    idx, cnt = compact(m)
+    out = {"tok": tok, "ent": H, "ent_norm": Hn, "gap": gap, "mask": m,
+           "llm_idx": idx, "llm_count": cnt}
+    if seq_len is not None:
+        out["llm_span"], out["llm_row_off"] = spans(idx, seq_len, kv_len)
+    return out

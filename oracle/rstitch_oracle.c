@@ -1,0 +1,201 @@
+/*
+ * CPU oracle for the R-Stitch routing decision.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, fp64 statement of what the path computes, written from the
+ * paper's definitions.  It shares no code, header, table or constant with the
+ * CUDA library; only tests, the smoke check and the benchmark's CPU-baseline
+ * leg may call it.  Inputs are the same bf16 bit patterns the GPU consumes,
+ * widened exactly to double.
+ *
+ * Every function below is pinned by CPU tests against closed forms, textbook
+ * special cases, an extended-precision brute force and a library log-softmax.
+ * The paper prints no numeric entropy, token id or mask for any input, so
+ * agreement with the paper's own numbers is "parity unpinned": only the
+ * definition (Eq. 1), the rule (Eq. 2, Algorithm 1) and the span arithmetic
+ * (Algorithm 1, prefill branch) are pinned.
+ *
+ * The vocabulary loop of the logit step is split over OpenMP threads; that
+ * is the only parallelism, and no blocking, fusion or reordering is applied.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* bf16 -> double, exact: bf16 is the top 16 bits of an IEEE float32. */
+static double bf16_to_double(uint16_t b)
+{
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/*
+ * Logits of one row (Section 3.1: the active model's last linear map turns
+ * the final hidden state into the distribution p_t over V entries):
+ *     z[v] = sum_{k=0}^{d-1} hidden[k] * W_head[v, k],   k ascending.
+ * W_head is row-major [V, d].
+ */
+void oracle_logits_row(const uint16_t *hidden_row, const uint16_t *w_head,
+                       int d, int V, double *z)
+{
+    double *h = (double *)malloc((size_t)d * sizeof(double));
+    for (int k = 0; k < d; ++k) h[k] = bf16_to_double(hidden_row[k]);
+#pragma omp parallel for schedule(static)
+    for (int v = 0; v < V; ++v) {
+        const uint16_t *wv = w_head + (size_t)v * (size_t)d;
+        double acc = 0.0;
+        for (int k = 0; k < d; ++k) acc += h[k] * bf16_to_double(wv[k]);
+        z[v] = acc;
+    }
+    free(h);
+}
+
+/*
+ * Greedy token (Section 3.1, y_t; greedy reading) and the top-2 logit gap.
+ * tok = lowest index attaining the maximum, NaN logits ignored; 0 if every
+ * logit is NaN.  gap = z[tok] - max_{v != tok} z[v] (0 on an exact tie).
+ */
+void oracle_greedy(const double *z, int V, int32_t *tok, double *gap)
+{
+    int best = -1;
+    for (int v = 0; v < V; ++v) {
+        if (isnan(z[v])) continue;
+        if (best < 0 || z[v] > z[best]) best = v;
+    }
+    if (best < 0) { *tok = 0; *gap = NAN; return; }
+    double second = -INFINITY;
+    for (int v = 0; v < V; ++v) {
+        if (v == best || isnan(z[v])) continue;
+        if (z[v] > second) second = z[v];
+    }
+    *tok = (int32_t)best;
+    *gap = z[best] - second;
+}
+
+/*
+ * Softmax entropy in nats (numerator of Eq. 1), two passes, no online trick:
+ *     m      = max_v z[v]
+ *     lse    = m + log sum_v exp(z[v] - m)
+ *     logp_v = z[v] - lse,  p_v = exp(logp_v)
+ *     H      = - sum_v p_v * logp_v        (a term is 0 when p_v underflows to 0)
+ * NaN logits propagate to a NaN entropy.
+ */
+double oracle_entropy_nats(const double *z, int V)
+{
+    double m = -INFINITY;
+    for (int v = 0; v < V; ++v) {
+        if (isnan(z[v])) return NAN;
+        if (z[v] > m) m = z[v];
+    }
+    double sum = 0.0;
+    for (int v = 0; v < V; ++v) sum += exp(z[v] - m);
+    double lse = m + log(sum);
+    double H = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double logp = z[v] - lse;
+        double p = exp(logp);
+        if (p > 0.0) H -= p * logp;
+    }
+    return H;
+}
+
+/* Eq. 1 in full: entropy divided by log V, a value in [0, 1]. */
+double oracle_entropy_normalized(const double *z, int V)
+{
+    return oracle_entropy_nats(z, V) / log((double)V);
+}
+
+/*
+ * Switching predicate (Eq. 2; Algorithm 1, "if H_t > tau"): strict.  On the
+ * SLM head 1 means hand the step to the LLM; on the LLM head 1 means stay on
+ * the LLM and 0 means return to the SLM.  A NaN entropy routes to the LLM.
+ */
+uint8_t oracle_rule(double H, double tau)
+{
+    if (isnan(H)) return 1;
+    return (H > tau) ? 1 : 0;
+}
+
+/*
+ * Head + entropy + greedy token for R rows.
+ *   hidden  bf16 bits, row-major [n_src, d]; row r reads hidden[row_idx[r]]
+ *           when row_idx != NULL, else hidden[r].
+ *   outputs per row: tok, H (nats), H / log V, top-2 gap.
+ */
+void oracle_head_rows(const uint16_t *hidden, const int32_t *row_idx,
+                      const uint16_t *w_head, int R, int d, int V,
+                      int32_t *tok, double *H_nats, double *H_norm, double *gap)
+{
+    double *z = (double *)malloc((size_t)V * sizeof(double));
+    for (int r = 0; r < R; ++r) {
+        size_t src = row_idx ? (size_t)row_idx[r] : (size_t)r;
+        oracle_logits_row(hidden + src * (size_t)d, w_head, d, V, z);
+        oracle_greedy(z, V, &tok[r], &gap[r]);
+        H_nats[r] = oracle_entropy_nats(z, V);
+        H_norm[r] = oracle_entropy_normalized(z, V);
+    }
+    free(z);
+}
+
+/*
+ * Per-sequence mask.  Without row_seq, sequence b is decided by row b
+ * (B == R).  With row_seq (int32 [R], non-decreasing sequence ids), the rows
+ * of one sequence are one stitched span run through a prefill, which yields
+ * one (p_t, y_t) at the end of the span (Algorithm 1, prefill branch): the
+ * decision row of a sequence is its last row.  Sequences without rows get 0.
+ */
+void oracle_mask(const double *H_nats, const int32_t *row_seq, int R, int B,
+                 double tau, uint8_t *mask)
+{
+    for (int b = 0; b < B; ++b) mask[b] = 0;
+    if (!row_seq) {
+        for (int b = 0; b < B && b < R; ++b) mask[b] = oracle_rule(H_nats[b], tau);
+        return;
+    }
+    for (int r = 0; r < R; ++r) {
+        int last = (r == R - 1) || (row_seq[r + 1] != row_seq[r]);
+        if (last && row_seq[r] >= 0 && row_seq[r] < B)
+            mask[row_seq[r]] = oracle_rule(H_nats[r], tau);
+    }
+}
+
+/* Ordered compaction: ascending list of b with mask[b] != 0, and its length. */
+void oracle_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count)
+{
+    int32_t n = 0;
+    for (int b = 0; b < B; ++b)
+        if (mask[b]) idx[n++] = (int32_t)b;
+    *count = n;
+}
+
+/*
+ * Stitched-span lengths of the routed sequences (Algorithm 1, prefill branch:
+ * the model that takes over prefills (x + y)[L:], i.e. |x + y| - L tokens) and
+ * their exclusive prefix sum, the row offsets of the catch-up batch;
+ * row_off[count] is the total number of rows.
+ */
+void oracle_spans(const int32_t *idx, int32_t count, const int32_t *seq_len,
+                  const int32_t *kv_len, int32_t *span, int32_t *row_off)
+{
+    int32_t acc = 0;
+    for (int32_t j = 0; j < count; ++j) {
+        span[j] = seq_len[idx[j]] - kv_len[idx[j]];
+        row_off[j] = acc;
+        acc += span[j];
+    }
+    row_off[count] = acc;
+}
