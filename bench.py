@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the R-Stitch routing-decision path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole hot path (LM-head contraction, entropy, greedy token, threshold
+rule, ordered compaction, stitched-span lengths) over one synthetic batch.  The default workload
+is the SLM head at batch 1 (d = 1536, V = 151936), the configuration the metric is quoted on.
+With N > 1 (one process per GPU under torch.distributed.run) every rank decides its own
+sequences against a replicated head: the path shards by rows with no data-path collective, so
+scaling is weak and the value is the sum over ranks divided by the slowest rank's time.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import rstitch_inputs as gen
+
+METRIC = "routing decisions/sec (fused head+entropy+route) and achieved HBM GB/s vs peak"
+UNIT = "decisions/s"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
+
+BENCH_WORKLOADS = {
+    "c2_slm_b1": ("c2_slm_b1",), "c3_llm_b1": ("c3_llm_b1",), "c3_llm_b4": ("c3_llm_b4",),
+    "c3_llm_b16": ("c3_llm_b16",), "c4_slm_b64": ("c4_slm_b64",),
+    "c4_batched": ("c4_slm_b64", "c4_llm_b64"), "c5_catchup": ("c5_catchup",), "c1_tiny": ("c1_tiny",),
+}
+
+
+# ------------------------------------------------------------------------------------------
+# clocks: read-only NVML polling during the timed region
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting",
+               0x100: "display_clock_setting", 0x10: "sync_boost"}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reason_bits, self.power = [], 0, []
+        self.sm_max = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+        self.period = period_s
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2.0)
+
+    def summary(self) -> dict:
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["unavailable"]}
+        reasons = sorted(name for bit, name in self.REASONS.items() if self.reason_bits & bit)
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.sm_max, "reasons": reasons,
+                "samples": len(self.samples),
+                "power_w_max": round(max(self.power), 1) if self.power else None}
+
+
+def visible_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def measured_peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            p = json.load(open(path))
+            return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                    "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    "source": "measured"}
+        except Exception:
+            pass
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+            "bf16_tflops_sustained": FALLBACK_BF16_TFLOPS_SUSTAINED, "source": "fallback"}
+
+
+def recorded_traffic(workload: str):
+    """DRAM bytes per launch of the dominant kernel from a committed ncu summary, if there is one."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        return json.load(open(path)).get(workload)
+    except Exception:
+        return None
+
+
+# ------------------------------------------------------------------------------------------
+# workload state
+# ------------------------------------------------------------------------------------------
+def build_batches(names, n_rot: int, rank: int):
+    """Host-side synthetic inputs: per head its W bits and n_rot rotating hidden batches."""
+    heads = []
+    for name in names:
+        w = gen.WORKLOADS[name]
+        w_bits = gen.make_w_head(w)
+        batches = []
+        for i in range(n_rot):
+            step = rank * 100003 + i
+            if w.span_max > 1:
+                k = gen.make_spans(w, step)
+                R = int(k.sum())
+                row_seq = np.repeat(np.arange(w.B, dtype=np.int32), k)
+                hid, _ = gen.make_hidden(w, w_bits, step, rows=R)
+                seq_len, kv_len = gen.make_kv_state(w, step, span=k)
+            else:
+                R, row_seq = w.B, None
+                hid, _ = gen.make_hidden(w, w_bits, step)
+                seq_len, kv_len = gen.make_kv_state(w, step)
+            batches.append({"hid": hid, "R": R, "row_seq": row_seq, "seq_len": seq_len, "kv_len": kv_len})
+        heads.append({"w": w, "w_bits": w_bits, "batches": batches})
+    return heads
+
+
+def run_reference(args, names) -> dict:
+    """The oracle as it stands, on the host cores, same metric / config."""
+    import oracle
+    oracle.build()
+    heads = build_batches(names, max(2, min(4, args.steps)), 0)
+    # a step is a bounded sample of the workload: at most `sample_rows` rows of each head's batch
+    sample_rows = 8 if sum(h["batches"][0]["R"] for h in heads) > 16 else None
+
+    def one_step(i):
+        rows = 0
+        for h in heads:
+            b = h["batches"][i % len(h["batches"])]
+            hid = b["hid"] if sample_rows is None else b["hid"][:sample_rows]
+            oracle.route(hid, h["w_bits"], h["w"].tau_nats)
+            rows += hid.shape[0]
+        return rows
+    for i in range(args.warmup):
+        one_step(i)
+    t0 = time.perf_counter()
+    rows = 0
+    for i in range(args.steps):
+        rows += one_step(i)
+    dt = time.perf_counter() - t0
+    value = rows / dt
+    sample = ("every row of each step" if sample_rows is None else
+              "first %d rows of each head's batch per step" % sample_rows)
+    w0 = heads[0]["w"]
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "B": w0.B, "d": w0.d, "V": w0.V},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main() -> int:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="c2_slm_b1", choices=sorted(BENCH_WORKLOADS))
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="rstitch_args_t.flags (testing)")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    names = BENCH_WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        args.steps = 8 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        print(json.dumps(run_reference(args, names)), flush=True)
+        return 0
+
+    import torch
+    import paper_2507_17307_b200 as rs
+    from paper_2507_17307_b200 import build as rs_build
+    if rank == 0:
+        rs_build.build_library()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    rs.lib()
+
+    heavy = args.workload in ("c5_catchup",)
+    K = args.steps if args.steps is not None else (64 if heavy else (2048 if args.workload == "c4_batched" else 8192))
+    Wm = args.warmup if args.warmup is not None else (3 if heavy else 64)
+    Wm = max(Wm, 3)
+    n_rot = 2 if heavy else 8
+
+    heads = build_batches(names, n_rot, rank)
+    dev = torch.device("cuda", local_rank)
+
+    def bf16_dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    def i32_dev(a):
+        return None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+
+    stream = torch.cuda.current_stream()
+    handles, prepared = [], [[] for _ in range(n_rot)]
+    prev_out = [None] * n_rot
+    algo_bytes = 0
+    flops = 0.0
+    for hi, h in enumerate(heads):
+        w = h["w"]
+        Rmax = max(b["R"] for b in h["batches"])
+        hd = rs.Handle(max(Rmax, 64), w.d, w.V)
+        handles.append(hd)
+        w_dev = bf16_dev(h["w_bits"])
+        h["w_dev"] = w_dev
+        algo_bytes += w.V * w.d * 2
+        for i, b in enumerate(h["batches"]):
+            R = b["R"]
+            out = rs.RouteOutputs.allocate(R, w.B, dev, spans=True)
+            kw = dict(R=R, B=w.B, seq_len=i32_dev(b["seq_len"]), kv_len=i32_dev(b["kv_len"]),
+                      row_seq=i32_dev(b["row_seq"]), flags=args.flags, stream=stream)
+            if hi == 1:
+                # batched step: the LLM head runs on the subset the SLM head routed, count on device
+                kw.update(row_idx=prev_out[i].llm_idx, n_rows_dev=prev_out[i].llm_count)
+            prepared[i].append(rs.PreparedCall(hd, bf16_dev(b["hid"]), w_dev, w.tau_nats, out, **kw))
+            if hi == 0:
+                prev_out[i] = out
+        flops += 2.0 * np.mean([b["R"] for b in h["batches"]]) * w.d * w.V
+    w0 = heads[0]["w"]
+    rows_per_step = float(np.mean([b["R"] for b in heads[0]["batches"]]))
+    decisions_per_step = rows_per_step            # rows decided by the first head of the step
+
+    def step(i):
+        for call in prepared[i % n_rot]:
+            st = call.launch()
+            if st != 0:
+                raise rs.RstitchError(st, "rstitch_route_ex")
+
+    for i in range(Wm):
+        step(i)
+    torch.cuda.synchronize()
+    for hd in handles:
+        rs.last_status(hd)                       # clears the launch counters
+
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(visible_gpu_index(local_rank)) as clocks:
+        ev0.record(stream)
+        for i in range(K):
+            step(i)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = sum(rs.last_status(hd)["launches"] for hd in handles)
+    stat_timeouts = 0
+
+    # end to end: per-step host buffers through rstitch_route_host (first head of the step)
+    h0 = heads[0]
+    e2e = None
+    if h0["batches"][0]["row_seq"] is None:
+        B = w0.B
+        pinned = [torch.from_numpy(b["hid"].view(np.int16)).view(torch.bfloat16).pin_memory()
+                  for b in h0["batches"]]
+        host_out = {"tok": torch.empty(B, dtype=torch.int32).pin_memory(),
+                    "ent": torch.empty(B, dtype=torch.float32).pin_memory(),
+                    "mask": torch.empty(B, dtype=torch.uint8).pin_memory(),
+                    "llm_idx": torch.empty(B, dtype=torch.int32).pin_memory(),
+                    "llm_count": torch.empty(1, dtype=torch.int32).pin_memory()}
+        Ke = min(K, 2048)
+        for i in range(3):
+            rs.route_host(handles[0], pinned[i % n_rot], h0["w_dev"], w0.tau_nats, host_out, stream)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for i in range(Ke):
+            rs.route_host(handles[0], pinned[i % n_rot], h0["w_dev"], w0.tau_nats, host_out, stream)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        e2e = {"seconds": e2e_s, "steps": Ke, "h2d": B * w0.d * 2, "d2h": B * 13 + 4}
+
+    # max over ranks
+    if dist is not None:
+        t = torch.tensor([ms, e2e["seconds"] if e2e else 0.0], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t[0].item())
+        if e2e:
+            e2e["seconds"] = float(t[1].item())
+        lt = torch.tensor([launches], dtype=torch.int64, device=dev)
+        dist.all_reduce(lt)
+        launches = int(lt.item())
+
+    if rank == 0:
+        peaks = measured_peaks()
+        sec = ms / 1e3
+        value = world * decisions_per_step * K / sec
+        per_launch_s = sec / K
+        tensor_bound = rows_per_step >= 256
+        if tensor_bound:
+            achieved = flops / per_launch_s / 1e12
+            peak = peaks["bf16_tflops_sustained"] if sec > 1.0 else peaks["bf16_tflops"]
+            roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "traffic": recorded_traffic(args.workload),
+                    "peak_source": "of " + peaks["source"],
+                    "hbm_gbs": algo_bytes / per_launch_s / 1e9}
+        else:
+            achieved = algo_bytes / per_launch_s / 1e9
+            roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": recorded_traffic(args.workload),
+                    "peak_source": "of " + peaks["source"], "frac_of_8tbs_nominal": achieved / 8000.0,
+                    "tflops": flops / per_launch_s / 1e12}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "B": w0.B, "rows_per_step": rows_per_step, "d": w0.d,
+                       "V": w0.V, "tau_nats": w0.tau_nats, "heads": list(names),
+                       "path": [rs.path_name(int(rows_per_step), h["w"].d, h["w"].V, args.flags) for h in heads],
+                       "l2": "inputs larger than L2: each step streams the whole W_head (%.0f MB); "
+                             "hidden rotates over %d buffers" % (algo_bytes / 1e6, n_rot),
+                       "parallelism": "dp%d (rows sharded, head replicated, no collective)" % world},
+            "roofline": roof, "clocks": clocks.summary(), "gpu_launches": launches,
+            "algorithmic_bytes_per_step": algo_bytes, "flops_per_step": flops,
+        }
+        if e2e:
+            line["e2e"] = {"value": world * w0.B * e2e["steps"] / e2e["seconds"], "unit": UNIT,
+                           "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                           "steps": e2e["steps"],
+                           "note": "rstitch_route_host: pinned hidden in, tok/ent/mask/llm_idx/llm_count out, "
+                                   "stream synchronised every step; W_head resident"}
+        else:
+            line["e2e"] = None
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            budget, t0, rows, n = 12.0, time.perf_counter(), 0, 0
+            sample_rows = 8 if rows_per_step > 16 else None
+            while time.perf_counter() - t0 < budget and n < 4096:
+                for h in heads:
+                    b = h["batches"][n % n_rot]
+                    hid = b["hid"] if sample_rows is None else b["hid"][:sample_rows]
+                    oracle.route(hid, h["w_bits"], h["w"].tau_nats)
+                rows += (heads[0]["batches"][n % n_rot]["hid"].shape[0] if sample_rows is None else sample_rows)
+                n += 1
+            dt = time.perf_counter() - t0
+            line["cpu_baseline"] = {"value": rows / dt, "unit": UNIT, "cores": oracle.num_threads(),
+                                    "kind": "oracle",
+                                    "sample": "%d steps%s of the same batches, %.1f s" % (
+                                        n, "" if sample_rows is None else " (first %d rows each)" % sample_rows, dt)}
+        print(json.dumps(line), flush=True)
+    for hd in handles:
+        hd.destroy()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

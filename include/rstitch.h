@@ -1,0 +1,179 @@
+/*
+ * rstitch.h -- C ABI of the R-Stitch routing-decision library (sm_100a).
+ *
+ * One call evaluates, for every active sequence of a hybrid SLM/LLM decode
+ * step, the tail of the model forward and the routing decision of the paper:
+ *
+ *   S1  logits   z[r,v] = sum_k hidden[r,k] * W_head[v,k]      (Section 3.1: p_t = f(y_{1:t-1}))
+ *   S2  entropy  H[r]   = -sum_v p_v ln p_v,  p = softmax(z_r) (Eq. 1, numerator; nats)
+ *   S3  token    tok[r] = argmax_v z[r,v], lowest index on ties (Section 3.1, y_t; greedy reading)
+ *   S4  rule     mask[b] = H[decision row of b] > tau           (Eq. 2; Algorithm 1 "if H_t > tau")
+ *   S5  compaction  llm_idx = ascending {b : mask[b] = 1}, llm_count = |llm_idx|
+ *   S6  spans    llm_span[j] = seq_len[llm_idx[j]] - kv_len[llm_idx[j]]  (Algorithm 1, prefill branch)
+ *                llm_row_off = exclusive prefix sum of llm_span, llm_row_off[llm_count] = total rows
+ *
+ * On the SLM head mask = 1 hands the step to the LLM (the SLM token is
+ * discarded by the caller); on the LLM head mask = 1 keeps the LLM active and
+ * mask = 0 returns control to the SLM.  Logits are never written to memory.
+ *
+ * Units: ent_out and tau are in nats.  The paper's normalised threshold
+ * (Eq. 1 divides by ln V) is tau_nats = tau_paper * ln V; pass
+ * RSTITCH_TAU_NORMALIZED to have the library do that multiplication.
+ *
+ * Conventions
+ *  - Every entry point returns an int status (0 = RSTITCH_OK, < 0 = error) and
+ *    never throws, exits or traps.  Arguments are validated on the host before
+ *    anything is launched; a failed validation launches nothing.
+ *  - Unless a parameter says "host", pointers are DEVICE pointers owned by the
+ *    caller.  The library neither frees nor reallocates them.  Device pointers
+ *    must be 16-byte aligned (hidden, W_head) or naturally aligned (the rest).
+ *  - Calls are asynchronous on the given CUDA stream: outputs are valid once
+ *    that stream has been synchronised.  llm_count stays on the device so that
+ *    the next model's step can be enqueued without a host round trip.
+ *  - bf16 tensors are row-major with the contraction index k contiguous.
+ *  - Non-finite inputs: a row whose entropy is NaN is routed (mask = 1), its
+ *    token is the lowest index of the largest non-NaN logit (0 if none), and
+ *    the row is counted in rstitch_devstat_t.nan_rows.
+ */
+#ifndef RSTITCH_H_
+#define RSTITCH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------ */
+#define RSTITCH_OK                     0
+#define RSTITCH_ERR_INVALID_ARG      (-1)  /* null pointer, negative size, non-finite tau, bad flag mix */
+#define RSTITCH_ERR_BAD_ALIGN        (-2)  /* a pointer misses its alignment */
+#define RSTITCH_ERR_UNSUPPORTED_SHAPE (-3) /* d % 8 != 0, d < 8, V < 2, or a size above the handle's maxima */
+#define RSTITCH_ERR_CUDA             (-4)  /* a CUDA runtime or driver call failed */
+#define RSTITCH_ERR_WORKSPACE        (-5)  /* caller workspace too small or misaligned */
+#define RSTITCH_ERR_TIMEOUT          (-6)  /* a bounded device-side wait gave up (see rstitch_last_status) */
+
+/* ---- flags for rstitch_args_t.flags ------------------------------------ */
+#define RSTITCH_TAU_NORMALIZED   0x1u  /* tau is the paper's normalised threshold in [0,1]; multiplied by ln V */
+#define RSTITCH_PATH_GEMV        0x10u /* testing only: force the CUDA-core streaming kernel */
+#define RSTITCH_PATH_UMMA        0x20u /* testing only: force the tcgen05 tensor-core kernel */
+
+typedef struct rstitch_handle_s *rstitch_handle_t;
+
+/*
+ * Arguments of the extended call.  Zero-initialise, then fill.
+ *
+ *   hidden      bf16 [n_src, d]   final hidden states
+ *   W_head      bf16 [V, d]       LM-head weights (no bias)
+ *   R           rows evaluated (each gives tok_out[r], ent_out[r])
+ *   B           sequences decided (route_mask has B entries).  Without row_seq, B must equal R
+ *               and sequence b is decided by row b.
+ *   n_src       rows present in hidden (only used to bound row_idx; 0 means R)
+ *   row_idx     optional int32 [R]: row r reads hidden[row_idx[r]] -- the LLM head evaluated on the
+ *               compacted subset llm_idx of an earlier SLM call.  Out-of-range entries are not
+ *               dereferenced; they read row 0 and are counted in devstat.bad_row_idx.
+ *   row_seq     optional int32 [R], non-decreasing sequence ids in [0, B): the rows of one sequence are
+ *               one stitched span pushed through a prefill.  A prefill yields one (p_t, y_t), at the
+ *               end of the span (Algorithm 1, prefill branch), so sequence b is decided by its LAST
+ *               row; sequences without rows get mask 0.
+ *   n_rows_dev  optional device int32 [1]: the live row count (<= R), e.g. the llm_count of an earlier
+ *               call.  Rows r >= *n_rows_dev are skipped and their outputs left untouched; B is
+ *               clamped the same way.  Not allowed together with row_seq.
+ *   seq_len, kv_len   optional int32 [B] (both or neither): |x + y| and the KV-cache length L of the
+ *               model that takes over, per sequence.
+ *   tok_out     int32 [R];  ent_out float32 [R] (nats)
+ *   route_mask  uint8 [B];  llm_idx int32 [B] (entries >= llm_count are left untouched);
+ *   llm_count   int32 [1]
+ *   llm_span    optional int32 [B], llm_row_off optional int32 [B + 1] (required iff seq_len is given).
+ *               A routed sequence with span < 1 is counted in devstat.bad_span.
+ *   workspace   optional caller scratch of at least rstitch_workspace_bytes(R, d, V) bytes, 256-byte
+ *               aligned; NULL uses the handle's own.  Two calls in flight at once on different
+ *               streams must not share a workspace.
+ */
+typedef struct rstitch_args_s {
+    const void    *hidden;
+    const void    *W_head;
+    int32_t        R, B, d, V, n_src;
+    float          tau;
+    uint32_t       flags;
+    const int32_t *row_idx;
+    const int32_t *row_seq;
+    const int32_t *n_rows_dev;
+    const int32_t *seq_len;
+    const int32_t *kv_len;
+    int32_t       *tok_out;
+    float         *ent_out;
+    uint8_t       *route_mask;
+    int32_t       *llm_idx;
+    int32_t       *llm_count;
+    int32_t       *llm_span;
+    int32_t       *llm_row_off;
+    void          *workspace;
+    size_t         workspace_bytes;
+} rstitch_args_t;
+
+/* Device status word, accumulated since the handle was created or last read. */
+typedef struct rstitch_devstat_s {
+    uint32_t nan_rows;      /* rows whose entropy came out NaN (routed, see above) */
+    uint32_t bad_row_idx;   /* row_idx entries outside [0, n_src) */
+    uint32_t bad_span;      /* routed sequences with seq_len - kv_len < 1 */
+    uint32_t timeouts;      /* bounded device-side waits that gave up */
+    uint32_t timeout_site;  /* where the last one gave up (kernel-internal site id) */
+    uint32_t launches;      /* kernels launched through this handle */
+    uint32_t reserved[2];
+} rstitch_devstat_t;
+
+/*
+ * Basic form (the routing problem as the paper states it, batched): B rows, one decision per row,
+ * S1-S5.  Runs on the legacy default stream with a per-device internal handle that is created on
+ * first use (that first call allocates device memory).  B = 0 is valid and sets *llm_count = 0.
+ */
+int rstitch_route(const void *hidden /* bf16 [B,d] */, const void *W_head /* bf16 [V,d] */,
+                  int B, int d, int V, float tau /* nats */,
+                  int32_t *tok_out /* [B] */, float *ent_out /* [B], nats */,
+                  uint8_t *route_mask /* [B] */, int32_t *llm_idx /* [B] */,
+                  int32_t *llm_count /* [1] */);
+
+/* Extended form, same arithmetic: explicit handle, stream (a cudaStream_t passed as void*), row
+ * gather, multi-row spans, S6.  See rstitch_args_t. */
+int rstitch_route_ex(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_stream);
+
+/*
+ * Same decision as rstitch_route with HOST buffers for the per-step data: hidden_host (bf16 [B,d],
+ * ideally pinned) is copied to the device, the step runs, and tok/ent/mask/llm_idx/llm_count are
+ * copied back to the given host buffers; the call returns after the stream has been synchronised.
+ * W_head is a model weight and stays a device pointer.  Staging buffers live in the handle.
+ */
+int rstitch_route_host(rstitch_handle_t h, const void *hidden_host, const void *W_head_dev,
+                       int B, int d, int V, float tau,
+                       int32_t *tok_host, float *ent_host, uint8_t *mask_host,
+                       int32_t *llm_idx_host, int32_t *llm_count_host, void *cuda_stream);
+
+/* Handle: owns the scratch memory and the device status word for problems up to the given maxima on
+ * the current device.  rstitch_destroy(NULL) is a no-op. */
+int rstitch_create(rstitch_handle_t *out, int maxR, int max_d, int maxV);
+int rstitch_destroy(rstitch_handle_t h);
+
+/* Scratch bytes one call of that shape needs (0 for an unsupported shape). */
+size_t rstitch_workspace_bytes(int R, int d, int V);
+
+/* S5 alone: ordered compaction of a uint8 mask [B] into idx [B] and count [1] (warp ballot + prefix
+ * sums).  Needs no handle; scratch for very large B is taken from a per-device internal handle. */
+int rstitch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, void *cuda_stream);
+
+/* Synchronises the handle's last stream, copies the device status word to *out (host) and clears it.
+ * h = NULL reads the per-device internal handle behind rstitch_route / rstitch_compact.
+ * Returns RSTITCH_ERR_TIMEOUT if a bounded wait gave up since the last read. */
+int rstitch_last_status(rstitch_handle_t h, rstitch_devstat_t *out);
+
+/* Static, never NULL. */
+const char *rstitch_status_string(int status);
+
+/* Name of the kernel family a call of that shape takes: "gemv" or "umma" (static string). */
+const char *rstitch_path_name(int R, int d, int V, uint32_t flags);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RSTITCH_H_ */

@@ -1,0 +1,10 @@
+"""R-Stitch routing decision at the LM head, B200-native (sm_100a CUDA behind a C ABI).
+
+The Python layer only marshals arguments: every step of the path runs in the kernels of
+``librstitch.so``.  There is no CPU or PyTorch fallback; a missing library raises.
+"""
+from .binding import (  # noqa: F401
+    RstitchError, Handle, RouteOutputs, PreparedCall, lib, library_path, route, route_ex, route_host, compact,
+    last_status, workspace_bytes, status_string, path_name,
+    TAU_NORMALIZED, PATH_GEMV, PATH_UMMA,
+)

@@ -1,0 +1,287 @@
+"""ctypes binding of include/rstitch.h: same names, argument marshalling only.
+
+PyTorch appears here for device memory and streams; nothing is computed in Python.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "librstitch.so")
+_lib = None
+
+TAU_NORMALIZED = 0x1
+PATH_GEMV = 0x10
+PATH_UMMA = 0x20
+
+EXPORTS = [
+    "rstitch_route", "rstitch_route_ex", "rstitch_route_host", "rstitch_create", "rstitch_destroy",
+    "rstitch_workspace_bytes", "rstitch_compact", "rstitch_last_status", "rstitch_status_string",
+    "rstitch_path_name",
+]
+
+
+class RstitchError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %d (%s)" % (where, status, status_string(status)))
+
+
+class _Args(C.Structure):
+    _fields_ = [
+        ("hidden", C.c_void_p), ("W_head", C.c_void_p),
+        ("R", C.c_int32), ("B", C.c_int32), ("d", C.c_int32), ("V", C.c_int32), ("n_src", C.c_int32),
+        ("tau", C.c_float), ("flags", C.c_uint32),
+        ("row_idx", C.c_void_p), ("row_seq", C.c_void_p), ("n_rows_dev", C.c_void_p),
+        ("seq_len", C.c_void_p), ("kv_len", C.c_void_p),
+        ("tok_out", C.c_void_p), ("ent_out", C.c_void_p), ("route_mask", C.c_void_p),
+        ("llm_idx", C.c_void_p), ("llm_count", C.c_void_p),
+        ("llm_span", C.c_void_p), ("llm_row_off", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+    ]
+
+
+class DevStat(C.Structure):
+    _fields_ = [("nan_rows", C.c_uint32), ("bad_row_idx", C.c_uint32), ("bad_span", C.c_uint32),
+                ("timeouts", C.c_uint32), ("timeout_site", C.c_uint32), ("launches", C.c_uint32),
+                ("reserved", C.c_uint32 * 2)]
+
+    def as_dict(self):
+        return {k: int(getattr(self, k)) for k in
+                ("nan_rows", "bad_row_idx", "bad_span", "timeouts", "timeout_site", "launches")}
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def lib():
+    """The loaded C library.  Raises if it has not been built: there is no other path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(
+                "librstitch.so is missing (%s): build it with "
+                "`python -m paper_2507_17307_b200.build`; there is no fallback path" % _LIB_PATH)
+        L = C.CDLL(_LIB_PATH)
+        vp, i, f = C.c_void_p, C.c_int, C.c_float
+        L.rstitch_route.argtypes = [vp, vp, i, i, i, f, vp, vp, vp, vp, vp]
+        L.rstitch_route.restype = i
+        L.rstitch_route_ex.argtypes = [vp, C.POINTER(_Args), vp]
+        L.rstitch_route_ex.restype = i
+        L.rstitch_route_host.argtypes = [vp, vp, vp, i, i, i, f, vp, vp, vp, vp, vp, vp]
+        L.rstitch_route_host.restype = i
+        L.rstitch_create.argtypes = [C.POINTER(vp), i, i, i]
+        L.rstitch_create.restype = i
+        L.rstitch_destroy.argtypes = [vp]
+        L.rstitch_destroy.restype = i
+        L.rstitch_workspace_bytes.argtypes = [i, i, i]
+        L.rstitch_workspace_bytes.restype = C.c_size_t
+        L.rstitch_compact.argtypes = [vp, i, vp, vp, vp]
+        L.rstitch_compact.restype = i
+        L.rstitch_last_status.argtypes = [vp, C.POINTER(DevStat)]
+        L.rstitch_last_status.restype = i
+        L.rstitch_status_string.argtypes = [i]
+        L.rstitch_status_string.restype = C.c_char_p
+        L.rstitch_path_name.argtypes = [i, i, i, C.c_uint32]
+        L.rstitch_path_name.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().rstitch_status_string(int(status)).decode()
+
+
+def path_name(R: int, d: int, V: int, flags: int = 0) -> str:
+    return lib().rstitch_path_name(int(R), int(d), int(V), int(flags)).decode()
+
+
+def workspace_bytes(R: int, d: int, V: int) -> int:
+    return int(lib().rstitch_workspace_bytes(int(R), int(d), int(V)))
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) or None
+
+
+class Handle:
+    """rstitch_create / rstitch_destroy."""
+
+    def __init__(self, maxR: int, max_d: int, maxV: int):
+        h = C.c_void_p()
+        st = lib().rstitch_create(C.byref(h), int(maxR), int(max_d), int(maxV))
+        if st != 0:
+            raise RstitchError(st, "rstitch_create")
+        self._h = h
+
+    @property
+    def ptr(self):
+        return self._h
+
+    def destroy(self):
+        if self._h is not None and self._h.value:
+            lib().rstitch_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+@dataclass
+class RouteOutputs:
+    """Device buffers one call writes."""
+    tok: "object"
+    ent: "object"
+    mask: "object"
+    llm_idx: "object"
+    llm_count: "object"
+    llm_span: "object" = None
+    llm_row_off: "object" = None
+
+    @staticmethod
+    def allocate(R: int, B: int, device, spans: bool = False) -> "RouteOutputs":
+        import torch
+        o = RouteOutputs(
+            tok=torch.full((max(R, 1),), -1, dtype=torch.int32, device=device),
+            ent=torch.full((max(R, 1),), -1.0, dtype=torch.float32, device=device),
+            mask=torch.full((max(B, 1),), 255, dtype=torch.uint8, device=device),
+            llm_idx=torch.full((max(B, 1),), -1, dtype=torch.int32, device=device),
+            llm_count=torch.full((1,), -1, dtype=torch.int32, device=device))
+        if spans:
+            o.llm_span = torch.full((max(B, 1),), -1, dtype=torch.int32, device=device)
+            o.llm_row_off = torch.full((B + 1,), -1, dtype=torch.int32, device=device)
+        return o
+
+
+def route(hidden, W_head, tau: float, out: Optional[RouteOutputs] = None) -> RouteOutputs:
+    """rstitch_route: B rows, one decision per row, on the legacy default stream."""
+    B, d = int(hidden.shape[0]), int(hidden.shape[1])
+    V = int(W_head.shape[0])
+    if out is None:
+        out = RouteOutputs.allocate(B, B, hidden.device)
+    st = lib().rstitch_route(_ptr(hidden), _ptr(W_head), B, d, V, float(tau), _ptr(out.tok), _ptr(out.ent),
+                             _ptr(out.mask), _ptr(out.llm_idx), _ptr(out.llm_count))
+    if st != 0:
+        raise RstitchError(st, "rstitch_route")
+    return out
+
+
+def route_ex(handle: Handle, hidden, W_head, tau: float, *, R: Optional[int] = None,
+             B: Optional[int] = None, row_idx=None, row_seq=None, n_rows_dev=None, seq_len=None,
+             kv_len=None, flags: int = 0, stream=None, out: Optional[RouteOutputs] = None,
+             workspace=None, check: bool = True):
+    """rstitch_route_ex.  Returns the outputs (or the status when check=False)."""
+    n_src, d = int(hidden.shape[0]), int(hidden.shape[1])
+    V = int(W_head.shape[0])
+    if R is None:
+        R = int(row_idx.shape[0]) if row_idx is not None else n_src
+    if B is None:
+        B = R
+    if out is None:
+        out = RouteOutputs.allocate(R, B, hidden.device, spans=seq_len is not None)
+    a = _Args()
+    a.hidden, a.W_head = _ptr(hidden), _ptr(W_head)
+    a.R, a.B, a.d, a.V, a.n_src = R, B, d, V, n_src
+    a.tau, a.flags = float(tau), int(flags)
+    a.row_idx, a.row_seq, a.n_rows_dev = _ptr(row_idx), _ptr(row_seq), _ptr(n_rows_dev)
+    a.seq_len, a.kv_len = _ptr(seq_len), _ptr(kv_len)
+    a.tok_out, a.ent_out, a.route_mask = _ptr(out.tok), _ptr(out.ent), _ptr(out.mask)
+    a.llm_idx, a.llm_count = _ptr(out.llm_idx), _ptr(out.llm_count)
+    a.llm_span, a.llm_row_off = _ptr(out.llm_span), _ptr(out.llm_row_off)
+    if workspace is not None:
+        a.workspace, a.workspace_bytes = _ptr(workspace), int(workspace.numel() * workspace.element_size())
+    st = lib().rstitch_route_ex(handle.ptr, C.byref(a), _stream_ptr(stream))
+    if not check:
+        return st
+    if st != 0:
+        raise RstitchError(st, "rstitch_route_ex")
+    return out
+
+
+class PreparedCall:
+    """A filled rstitch_args_t kept alive with its tensors, so that a step loop pays one C call
+    per step and no Python marshalling.  launch() is rstitch_route_ex with those arguments."""
+
+    def __init__(self, handle: Handle, hidden, W_head, tau: float, out: RouteOutputs, *, R=None, B=None,
+                 row_idx=None, row_seq=None, n_rows_dev=None, seq_len=None, kv_len=None, flags=0,
+                 stream=None):
+        n_src, d = int(hidden.shape[0]), int(hidden.shape[1])
+        if R is None:
+            R = int(row_idx.shape[0]) if row_idx is not None else n_src
+        if B is None:
+            B = R
+        a = _Args()
+        a.hidden, a.W_head = _ptr(hidden), _ptr(W_head)
+        a.R, a.B, a.d, a.V, a.n_src = R, B, d, int(W_head.shape[0]), n_src
+        a.tau, a.flags = float(tau), int(flags)
+        a.row_idx, a.row_seq, a.n_rows_dev = _ptr(row_idx), _ptr(row_seq), _ptr(n_rows_dev)
+        a.seq_len, a.kv_len = _ptr(seq_len), _ptr(kv_len)
+        a.tok_out, a.ent_out, a.route_mask = _ptr(out.tok), _ptr(out.ent), _ptr(out.mask)
+        a.llm_idx, a.llm_count = _ptr(out.llm_idx), _ptr(out.llm_count)
+        a.llm_span, a.llm_row_off = _ptr(out.llm_span), _ptr(out.llm_row_off)
+        self._keep = (handle, hidden, W_head, out, row_idx, row_seq, n_rows_dev, seq_len, kv_len)
+        self._args = a
+        self._ref = C.byref(a)
+        self._h = handle.ptr
+        self._stream = _stream_ptr(stream)
+        self._fn = lib().rstitch_route_ex
+        self.out = out
+
+    def launch(self) -> int:
+        return self._fn(self._h, self._ref, self._stream)
+
+
+def route_host(handle: Handle, hidden_host, W_head_dev, tau: float, host_out: dict, stream=None):
+    """rstitch_route_host: per-step data in host buffers (torch CPU tensors, ideally pinned).
+
+    host_out holds CPU tensors 'tok' int32 [B], 'ent' float32 [B], 'mask' uint8 [B],
+    'llm_idx' int32 [B], 'llm_count' int32 [1]; returns after the stream is synchronised.
+    """
+    B, d = int(hidden_host.shape[0]), int(hidden_host.shape[1])
+    V = int(W_head_dev.shape[0])
+    st = lib().rstitch_route_host(handle.ptr, _ptr(hidden_host), _ptr(W_head_dev), B, d, V, float(tau),
+                                  _ptr(host_out["tok"]), _ptr(host_out["ent"]), _ptr(host_out["mask"]),
+                                  _ptr(host_out["llm_idx"]), _ptr(host_out["llm_count"]),
+                                  _stream_ptr(stream))
+    if st != 0:
+        raise RstitchError(st, "rstitch_route_host")
+    return host_out
+
+
+def compact(mask, idx=None, count=None, stream=None):
+    """rstitch_compact: (llm_idx int32 [B], llm_count int32 [1]) of a uint8 device mask."""
+    import torch
+    B = int(mask.shape[0])
+    if idx is None:
+        idx = torch.full((max(B, 1),), -1, dtype=torch.int32, device=mask.device)
+    if count is None:
+        count = torch.full((1,), -1, dtype=torch.int32, device=mask.device)
+    st = lib().rstitch_compact(_ptr(mask), B, _ptr(idx), _ptr(count), _stream_ptr(stream))
+    if st != 0:
+        raise RstitchError(st, "rstitch_compact")
+    return idx, count
+
+
+def last_status(handle: Optional[Handle] = None) -> dict:
+    """rstitch_last_status: device status word as a dict (adds 'status')."""
+    s = DevStat()
+    st = lib().rstitch_last_status(handle.ptr if handle is not None else None, C.byref(s))
+    if st not in (0, -6):
+        raise RstitchError(st, "rstitch_last_status")
+    out = s.as_dict()
+    out["status"] = st
+    return out

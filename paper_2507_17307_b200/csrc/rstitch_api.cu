@@ -1,0 +1,333 @@
+// C ABI of the routing-decision library: argument validation, handles, scratch memory and the
+// choice of kernel family.  All arithmetic of the path runs in the kernels; nothing here computes.
+#include "../../include/rstitch.h"
+#include "rstitch_kernels.cuh"
+
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+using namespace rstitch;
+
+static_assert(sizeof(DevStat) == sizeof(rstitch_devstat_t), "device status word layout");
+
+struct rstitch_handle_s {
+    int      device      = -1;
+    int      sm_count    = 0;
+    int      maxR = 0, max_d = 0, maxV = 0;
+    void    *ws          = nullptr;      // scratch: ticket + partials
+    size_t   ws_bytes    = 0;
+    DevStat *stat        = nullptr;      // device status word
+    int32_t *tile_counts = nullptr;      // scratch of the multi-block compaction
+    int      tile_cap    = 0;
+    // staging of rstitch_route_host
+    void    *st_hidden = nullptr;  size_t st_hidden_bytes = 0;
+    void    *st_out    = nullptr;  size_t st_out_bytes = 0;
+    cudaStream_t last_stream = nullptr;
+};
+
+namespace {
+
+constexpr int kMaxD = 16384;
+constexpr int kMaxRows = 16384;
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+size_t ws_bytes_for(int R)
+{
+    return kWsHeader + partials_bytes((size_t)(R > 0 ? R : 1), (size_t)kMaxSlices);
+}
+
+int shape_status(int R, int d, int V)
+{
+    if (R < 0) return RSTITCH_ERR_INVALID_ARG;
+    if (d < 8 || (d % 8) != 0 || d > kMaxD || V < 2 || R > kMaxRows) return RSTITCH_ERR_UNSUPPORTED_SHAPE;
+    return RSTITCH_OK;
+}
+
+int grow_handle(rstitch_handle_s *h, int R, int d, int V)
+{
+    size_t need = ws_bytes_for(R);
+    if (need > h->ws_bytes) {
+        if (h->ws) { if (cudaDeviceSynchronize() != cudaSuccess) return RSTITCH_ERR_CUDA; cudaFree(h->ws); h->ws = nullptr; h->ws_bytes = 0; }
+        if (cudaMalloc(&h->ws, need) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+        if (cudaMemset(h->ws, 0, kWsHeader) != cudaSuccess) return RSTITCH_ERR_CUDA;
+        h->ws_bytes = need;
+    }
+    if (R > h->maxR) h->maxR = R;
+    if (d > h->max_d) h->max_d = d;
+    if (V > h->maxV) h->maxV = V;
+    return RSTITCH_OK;
+}
+
+std::mutex       g_default_mutex;
+rstitch_handle_s *g_default[64] = {};
+
+// Per-device handle behind the entry points that take none; grows on demand.
+int default_handle(rstitch_handle_s **out, int R, int d, int V)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return RSTITCH_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_default_mutex);
+    if (!g_default[dev]) {
+        rstitch_handle_t h = nullptr;
+        int st = rstitch_create(&h, R > 64 ? R : 64, d, V);
+        if (st != RSTITCH_OK) return st;
+        g_default[dev] = h;
+    }
+    int st = grow_handle(g_default[dev], R, d, V);
+    if (st != RSTITCH_OK) return st;
+    *out = g_default[dev];
+    return RSTITCH_OK;
+}
+
+int validate(const rstitch_handle_s *h, const rstitch_args_t *a)
+{
+    if (!h || !a) return RSTITCH_ERR_INVALID_ARG;
+    int st = shape_status(a->R, a->d, a->V);
+    if (st != RSTITCH_OK) return st;
+    if (a->B < 0 || a->n_src < 0) return RSTITCH_ERR_INVALID_ARG;
+    if (!std::isfinite(a->tau)) return RSTITCH_ERR_INVALID_ARG;
+    if ((a->flags & RSTITCH_PATH_GEMV) && (a->flags & RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
+    if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
+    if (!a->llm_count) return RSTITCH_ERR_INVALID_ARG;
+    if (a->row_seq == nullptr && a->B != a->R) return RSTITCH_ERR_INVALID_ARG;
+    if (a->row_seq != nullptr && a->n_rows_dev != nullptr) return RSTITCH_ERR_INVALID_ARG;
+    if ((a->seq_len == nullptr) != (a->kv_len == nullptr)) return RSTITCH_ERR_INVALID_ARG;
+    if (a->seq_len && a->B > 0 && (!a->llm_span || !a->llm_row_off)) return RSTITCH_ERR_INVALID_ARG;
+    if (a->R > 0 && (!a->hidden || !a->W_head || !a->tok_out || !a->ent_out)) return RSTITCH_ERR_INVALID_ARG;
+    if (a->B > 0 && (!a->route_mask || !a->llm_idx)) return RSTITCH_ERR_INVALID_ARG;
+    if (!aligned(a->hidden, 16) || !aligned(a->W_head, 16)) return RSTITCH_ERR_BAD_ALIGN;
+    if (!aligned(a->tok_out, 4) || !aligned(a->ent_out, 4) || !aligned(a->llm_idx, 4) ||
+        !aligned(a->llm_count, 4) || !aligned(a->row_idx, 4) || !aligned(a->row_seq, 4) ||
+        !aligned(a->n_rows_dev, 4) || !aligned(a->seq_len, 4) || !aligned(a->kv_len, 4) ||
+        !aligned(a->llm_span, 4) || !aligned(a->llm_row_off, 4))
+        return RSTITCH_ERR_BAD_ALIGN;
+    if (a->workspace) {
+        if (!aligned(a->workspace, 256) || a->workspace_bytes < ws_bytes_for(a->R)) return RSTITCH_ERR_WORKSPACE;
+    } else if (a->R > h->maxR || a->d > h->max_d || a->V > h->maxV) {
+        return RSTITCH_ERR_UNSUPPORTED_SHAPE;
+    }
+    return RSTITCH_OK;
+}
+
+bool use_umma(int R, int d, int V, uint32_t flags)
+{
+    (void)R; (void)d; (void)V; (void)flags;
+    return false;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *rstitch_status_string(int status)
+{
+    switch (status) {
+        case RSTITCH_OK:                    return "ok";
+        case RSTITCH_ERR_INVALID_ARG:       return "invalid argument";
+        case RSTITCH_ERR_BAD_ALIGN:         return "misaligned pointer";
+        case RSTITCH_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case RSTITCH_ERR_CUDA:              return "CUDA call failed";
+        case RSTITCH_ERR_WORKSPACE:         return "workspace too small or misaligned";
+        case RSTITCH_ERR_TIMEOUT:           return "device-side wait timed out";
+        default:                            return "unknown status";
+    }
+}
+
+const char *rstitch_path_name(int R, int d, int V, uint32_t flags)
+{
+    return use_umma(R, d, V, flags) ? "umma" : "gemv";
+}
+
+size_t rstitch_workspace_bytes(int R, int d, int V)
+{
+    if (shape_status(R, d, V) != RSTITCH_OK) return 0;
+    return ws_bytes_for(R);
+}
+
+int rstitch_create(rstitch_handle_t *out, int maxR, int max_d, int maxV)
+{
+    if (!out) return RSTITCH_ERR_INVALID_ARG;
+    *out = nullptr;
+    int st = shape_status(maxR, max_d, maxV);
+    if (st != RSTITCH_OK) return st;
+    rstitch_handle_s *h = new (std::nothrow) rstitch_handle_s();
+    if (!h) return RSTITCH_ERR_CUDA;
+    bool ok = cudaGetDevice(&h->device) == cudaSuccess &&
+              cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) == cudaSuccess &&
+              cudaMalloc((void **)&h->stat, sizeof(DevStat)) == cudaSuccess &&
+              cudaMemset(h->stat, 0, sizeof(DevStat)) == cudaSuccess;
+    if (ok) ok = grow_handle(h, maxR, max_d, maxV) == RSTITCH_OK;
+    if (!ok) { cudaGetLastError(); rstitch_destroy(h); return RSTITCH_ERR_CUDA; }
+    *out = h;
+    return RSTITCH_OK;
+}
+
+int rstitch_destroy(rstitch_handle_t h)
+{
+    if (!h) return RSTITCH_OK;
+    cudaFree(h->ws); cudaFree(h->stat); cudaFree(h->tile_counts); cudaFree(h->st_hidden); cudaFree(h->st_out);
+    cudaGetLastError();
+    delete h;
+    return RSTITCH_OK;
+}
+
+int rstitch_route_ex(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_stream)
+{
+    int st = validate(h, a);
+    if (st != RSTITCH_OK) return st;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    h->last_stream = stream;
+
+    if (a->R == 0 || a->B == 0) {
+        // nothing to evaluate or nothing to decide: the compaction of an empty mask
+        if (cudaMemsetAsync(a->llm_count, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
+        if (a->seq_len && a->llm_row_off &&
+            cudaMemsetAsync(a->llm_row_off, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
+        if (a->R == 0) return RSTITCH_OK;
+    }
+
+    HeadArgs ha;
+    ha.hidden = a->hidden; ha.W = a->W_head; ha.R = a->R; ha.d = a->d; ha.V = a->V;
+    ha.n_src = a->n_src > 0 ? a->n_src : a->R;
+    ha.row_idx = a->row_idx; ha.n_rows_dev = a->n_rows_dev;
+
+    TailArgs ta;
+    ta.R = a->R; ta.B = a->B; ta.V = a->V;
+    ta.tau = (a->flags & RSTITCH_TAU_NORMALIZED) ? a->tau * logf((float)a->V) : a->tau;
+    ta.row_seq = a->row_seq; ta.seq_len = a->seq_len; ta.kv_len = a->kv_len;
+    ta.tok_out = a->tok_out; ta.ent_out = a->ent_out; ta.route_mask = a->route_mask;
+    ta.llm_idx = a->llm_idx; ta.llm_count = a->llm_count;
+    ta.llm_span = a->llm_span; ta.llm_row_off = a->llm_row_off;
+    ta.stat = h->stat;
+
+    Scratch sc = scratch_carve(a->workspace ? a->workspace : h->ws);
+    if (a->workspace) {
+        // caller scratch: the ticket must start at zero
+        if (cudaMemsetAsync(sc.ticket, 0, sizeof(unsigned), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
+    }
+    cudaError_t e = launch_head_gemv(ha, ta, sc, h->sm_count, stream);
+    if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    return RSTITCH_OK;
+}
+
+int rstitch_route(const void *hidden, const void *W_head, int B, int d, int V, float tau,
+                  int32_t *tok_out, float *ent_out, uint8_t *route_mask, int32_t *llm_idx,
+                  int32_t *llm_count)
+{
+    int st = shape_status(B, d, V);
+    if (st != RSTITCH_OK) return st;
+    rstitch_handle_s *h = nullptr;
+    st = default_handle(&h, B, d, V);
+    if (st != RSTITCH_OK) return st;
+    rstitch_args_t a;
+    std::memset(&a, 0, sizeof a);
+    a.hidden = hidden; a.W_head = W_head; a.R = B; a.B = B; a.d = d; a.V = V; a.n_src = B; a.tau = tau;
+    a.tok_out = tok_out; a.ent_out = ent_out; a.route_mask = route_mask; a.llm_idx = llm_idx;
+    a.llm_count = llm_count;
+    return rstitch_route_ex(h, &a, nullptr);
+}
+
+int rstitch_route_host(rstitch_handle_t h, const void *hidden_host, const void *W_head_dev,
+                       int B, int d, int V, float tau, int32_t *tok_host, float *ent_host,
+                       uint8_t *mask_host, int32_t *llm_idx_host, int32_t *llm_count_host,
+                       void *cuda_stream)
+{
+    if (!h) return RSTITCH_ERR_INVALID_ARG;
+    int st = shape_status(B, d, V);
+    if (st != RSTITCH_OK) return st;
+    if (!llm_count_host) return RSTITCH_ERR_INVALID_ARG;
+    if (B > 0 && (!hidden_host || !W_head_dev || !tok_host || !ent_host || !mask_host || !llm_idx_host))
+        return RSTITCH_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (B == 0) { *llm_count_host = 0; return RSTITCH_OK; }
+
+    // staging: hidden [B,d] bf16 | outputs packed as tok, ent, llm_idx (4 B each), count, mask
+    size_t hid_bytes = (size_t)B * d * 2;
+    size_t out_bytes = (size_t)B * 12 + 16 + (size_t)B;
+    if (hid_bytes > h->st_hidden_bytes) {
+        if (h->st_hidden) { cudaDeviceSynchronize(); cudaFree(h->st_hidden); h->st_hidden = nullptr; h->st_hidden_bytes = 0; }
+        if (cudaMalloc(&h->st_hidden, hid_bytes) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+        h->st_hidden_bytes = hid_bytes;
+    }
+    if (out_bytes > h->st_out_bytes) {
+        if (h->st_out) { cudaDeviceSynchronize(); cudaFree(h->st_out); h->st_out = nullptr; h->st_out_bytes = 0; }
+        if (cudaMalloc(&h->st_out, out_bytes) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+        h->st_out_bytes = out_bytes;
+    }
+    char *o = (char *)h->st_out;
+    int32_t *d_tok = (int32_t *)o;
+    float   *d_ent = (float *)(o + (size_t)B * 4);
+    int32_t *d_idx = (int32_t *)(o + (size_t)B * 8);
+    int32_t *d_cnt = (int32_t *)(o + (size_t)B * 12);
+    uint8_t *d_msk = (uint8_t *)(o + (size_t)B * 12 + 16);
+
+    if (cudaMemcpyAsync(h->st_hidden, hidden_host, hid_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    rstitch_args_t a;
+    std::memset(&a, 0, sizeof a);
+    a.hidden = h->st_hidden; a.W_head = W_head_dev; a.R = B; a.B = B; a.d = d; a.V = V; a.n_src = B; a.tau = tau;
+    a.tok_out = d_tok; a.ent_out = d_ent; a.route_mask = d_msk; a.llm_idx = d_idx; a.llm_count = d_cnt;
+    st = rstitch_route_ex(h, &a, cuda_stream);
+    if (st != RSTITCH_OK) return st;
+    // outputs are contiguous in the staging block: tok | ent | idx | count come back in one copy
+    bool ok = cudaMemcpyAsync(tok_host, d_tok, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+              cudaMemcpyAsync(ent_host, d_ent, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+              cudaMemcpyAsync(llm_idx_host, d_idx, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+              cudaMemcpyAsync(llm_count_host, d_cnt, 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+              cudaMemcpyAsync(mask_host, d_msk, (size_t)B, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+              cudaStreamSynchronize(stream) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    return RSTITCH_OK;
+}
+
+int rstitch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, void *cuda_stream)
+{
+    if (B < 0 || !count || (B > 0 && (!mask || !idx))) return RSTITCH_ERR_INVALID_ARG;
+    if (!aligned(idx, 4) || !aligned(count, 4)) return RSTITCH_ERR_BAD_ALIGN;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (B == 0) {
+        if (cudaMemsetAsync(count, 0, sizeof(int32_t), stream) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+        return RSTITCH_OK;
+    }
+    rstitch_handle_s *h = nullptr;
+    int st = default_handle(&h, 1, 8, 2);
+    if (st != RSTITCH_OK) return st;
+    int32_t *tiles = nullptr;
+    if (B > kCompactOneBlockMax) {
+        int n_tiles = (B + kCompactTile - 1) / kCompactTile;
+        std::lock_guard<std::mutex> lock(g_default_mutex);
+        if (n_tiles > h->tile_cap) {
+            if (h->tile_counts) { cudaDeviceSynchronize(); cudaFree(h->tile_counts); h->tile_counts = nullptr; h->tile_cap = 0; }
+            if (cudaMalloc((void **)&h->tile_counts, (size_t)n_tiles * 4) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+            h->tile_cap = n_tiles;
+        }
+        tiles = h->tile_counts;
+    }
+    h->last_stream = stream;
+    cudaError_t e = launch_compact(mask, B, idx, count, h->stat, tiles, stream);
+    if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    return RSTITCH_OK;
+}
+
+int rstitch_last_status(rstitch_handle_t h, rstitch_devstat_t *out)
+{
+    if (!out) return RSTITCH_ERR_INVALID_ARG;
+    if (!h) {
+        // the per-device handle behind rstitch_route / rstitch_compact
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+        std::lock_guard<std::mutex> lock(g_default_mutex);
+        h = g_default[dev];
+        if (!h) { std::memset(out, 0, sizeof *out); return RSTITCH_OK; }
+    }
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    if (cudaMemcpy(out, h->stat, sizeof(DevStat), cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemset(h->stat, 0, sizeof(DevStat)) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    return out->timeouts ? RSTITCH_ERR_TIMEOUT : RSTITCH_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,44 @@
+// Internal launch interfaces between the C ABI (rstitch_api.cu) and the kernel files.
+#pragma once
+#include "rstitch_tail.cuh"
+#include <cuda_runtime.h>
+
+namespace rstitch {
+
+constexpr int    kMaxSlices   = 1024;   // upper bound on vocabulary slices (partials per row)
+constexpr size_t kWsHeader    = 256;    // ticket counter lives in the first 256 bytes of the scratch
+
+// What the head kernels read.
+struct HeadArgs {
+    const void    *hidden;      // bf16 [n_src, d]
+    const void    *W;           // bf16 [V, d]
+    int            R, d, V, n_src;
+    const int32_t *row_idx;     // optional gather
+    const int32_t *n_rows_dev;  // optional live row count
+};
+
+struct Scratch {
+    unsigned *ticket;           // one counter, zero between launches
+    void     *partials;         // partials_bytes(R, n_slices)
+};
+
+__host__ inline Scratch scratch_carve(void *ws)
+{
+    Scratch s;
+    s.ticket   = (unsigned *)ws;
+    s.partials = (char *)ws + kWsHeader;
+    return s;
+}
+
+// CUDA-core streaming kernel: split-V GEMV for a handful of rows.
+cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch &s, int sm_count,
+                             cudaStream_t stream);
+
+// Stand-alone ordered compaction (S5).
+cudaError_t launch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, DevStat *stat,
+                           int32_t *block_counts /* scratch for B > one block's reach, or null */,
+                           cudaStream_t stream);
+constexpr int kCompactOneBlockMax = 1 << 16;
+constexpr int kCompactTile        = 4096;     // sequences per block in the multi-block form
+
+}  // namespace rstitch

@@ -1,0 +1,90 @@
+// Single-pass softmax statistics and their merge (device side only).
+//
+// For a set S of logits the kernels carry
+//     m = max z,   s = sum e^{z-m},   u = sum e^{z-m} (z-m),   (bv, bi) = greedy token
+// from which the entropy of Eq. 1 (in nats) is  H = ln s - u / s.
+// Two disjoint sets merge with M = max(m1, m2), a_i = e^{m_i - M}:
+//     s = a1 s1 + a2 s2,   u = a1 (u1 + (m1 - M) s1) + a2 (u2 + (m2 - M) s2).
+// The empty set is (m = -inf, s = 0, u = 0) and never produces inf - inf.
+#pragma once
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <limits.h>
+
+namespace rstitch {
+
+struct Stats {
+    float m, s, u, bv;
+    int   bi;
+};
+
+__device__ __forceinline__ Stats stats_empty()
+{
+    Stats t;
+    t.m = -CUDART_INF_F; t.s = 0.f; t.u = 0.f; t.bv = -CUDART_INF_F; t.bi = INT_MAX;
+    return t;
+}
+
+// Greedy token order: larger logit first, lower vocabulary index on ties.  NaN never wins.
+__device__ __forceinline__ void argmax_take(float &bv, int &bi, float v, int i)
+{
+    if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+}
+
+// Add one logit.
+__device__ __forceinline__ void stats_push(Stats &t, float z, int idx)
+{
+    argmax_take(t.bv, t.bi, z, idx);
+    float mn = fmaxf(t.m, z);                       // fmaxf ignores a NaN operand
+    float dm = (t.m == -CUDART_INF_F) ? 0.f : (t.m - mn);
+    float a  = __expf(dm);
+    float dz = z - mn;
+    float e  = __expf(dz);                          // NaN logit -> e = NaN -> s = NaN
+    t.u = a * (t.u + dm * t.s) + e * dz;
+    t.s = a * t.s + e;
+    t.m = mn;
+}
+
+// Merge b into a (a is the set with the lower vocabulary indices only by convention; the argmax
+// comparison is order-independent).
+__device__ __forceinline__ void stats_merge(Stats &a, const Stats &b)
+{
+    argmax_take(a.bv, a.bi, b.bv, b.bi);
+    float M  = fmaxf(a.m, b.m);
+    float da = (a.m == -CUDART_INF_F) ? 0.f : (a.m - M);
+    float db = (b.m == -CUDART_INF_F) ? 0.f : (b.m - M);
+    float ea = (a.m == -CUDART_INF_F) ? 0.f : __expf(da);
+    float eb = (b.m == -CUDART_INF_F) ? 0.f : __expf(db);
+    float s  = ea * a.s + eb * b.s;
+    float u  = ea * (a.u + da * a.s) + eb * (b.u + db * b.s);
+    a.m = M; a.s = s; a.u = u;
+}
+
+__device__ __forceinline__ Stats stats_shfl_xor(const Stats &t, int lane_mask)
+{
+    Stats o;
+    o.m  = __shfl_xor_sync(0xffffffffu, t.m, lane_mask);
+    o.s  = __shfl_xor_sync(0xffffffffu, t.s, lane_mask);
+    o.u  = __shfl_xor_sync(0xffffffffu, t.u, lane_mask);
+    o.bv = __shfl_xor_sync(0xffffffffu, t.bv, lane_mask);
+    o.bi = __shfl_xor_sync(0xffffffffu, t.bi, lane_mask);
+    return o;
+}
+
+// All lanes end with the merge of the 32 lanes' sets, in a fixed butterfly order.
+__device__ __forceinline__ void stats_warp_allmerge(Stats &t)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Stats p = stats_shfl_xor(t, o);
+        stats_merge(t, p);
+    }
+}
+
+// Entropy in nats from merged statistics.  s >= 1 for any non-empty finite set.
+__device__ __forceinline__ float stats_entropy(const Stats &t)
+{
+    return __logf(t.s) - t.u / t.s;
+}
+
+}  // namespace rstitch

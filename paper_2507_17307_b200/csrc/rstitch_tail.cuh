@@ -1,0 +1,175 @@
+// Cross-CTA finalisation of the head kernels and the routing tail (S2-S6), run by ONE thread
+// block: the block that drew the last ticket of a head kernel, or the single block of the
+// stand-alone compaction kernel.  No block ever waits on another, so nothing here can hang.
+#pragma once
+#include "rstitch_stats.cuh"
+#include <stdint.h>
+
+namespace rstitch {
+
+// Device status word; mirrors rstitch_devstat_t field by field.
+struct DevStat {
+    unsigned nan_rows, bad_row_idx, bad_span, timeouts, timeout_site, launches, r0, r1;
+};
+
+// Per-(row, slice) partial statistics in scratch memory, structure of arrays, [R][n_slices].
+struct Partials {
+    float *m, *s, *u, *bv;
+    int   *bi;
+};
+
+__host__ __device__ inline size_t partials_bytes(size_t R, size_t n_slices)
+{
+    size_t one = ((R * n_slices * 4 + 255) / 256) * 256;
+    return 5 * one;
+}
+
+__host__ __device__ inline Partials partials_carve(void *base, size_t R, size_t n_slices)
+{
+    size_t one = ((R * n_slices * 4 + 255) / 256) * 256;
+    char *p = (char *)base;
+    Partials q;
+    q.m  = (float *)(p);
+    q.s  = (float *)(p + one);
+    q.u  = (float *)(p + 2 * one);
+    q.bv = (float *)(p + 3 * one);
+    q.bi = (int *)(p + 4 * one);
+    return q;
+}
+
+__device__ __forceinline__ void partial_store(const Partials &P, size_t at, const Stats &t)
+{
+    P.m[at] = t.m; P.s[at] = t.s; P.u[at] = t.u; P.bv[at] = t.bv; P.bi[at] = t.bi;
+}
+
+__device__ __forceinline__ Stats partial_load(const Partials &P, size_t at)
+{
+    Stats t;                     // written by other blocks of this launch: bypass L1
+    t.m = __ldcg(P.m + at); t.s = __ldcg(P.s + at); t.u = __ldcg(P.u + at);
+    t.bv = __ldcg(P.bv + at); t.bi = __ldcg(P.bi + at);
+    return t;
+}
+
+struct TailArgs {
+    int R, B;                    // rows evaluated, sequences decided (already clamped to the live count)
+    int V;
+    float tau;                   // nats
+    const int32_t *row_seq;      // optional [R]
+    const int32_t *seq_len, *kv_len;   // optional [B]
+    int32_t *tok_out;            // [R]
+    float   *ent_out;            // [R]
+    uint8_t *route_mask;         // [B]
+    int32_t *llm_idx, *llm_count;
+    int32_t *llm_span, *llm_row_off;   // optional
+    DevStat *stat;
+};
+
+// Merge the n_slices partials of every row in a fixed order (lanes stride over slices, then a
+// butterfly), write ent_out / tok_out.  One warp per row.
+__device__ inline void tail_finalize_rows(const Partials &P, int n_slices, const TailArgs &a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int r = warp; r < a.R; r += nwarps) {
+        Stats t = stats_empty();
+        for (int c = lane; c < n_slices; c += 32) {
+            Stats p = partial_load(P, (size_t)r * n_slices + c);
+            stats_merge(t, p);
+        }
+        stats_warp_allmerge(t);
+        if (lane == 0) {
+            float H = logf(t.s) - t.u / t.s;
+            if (H < 0.f) H = 0.f;                      // rounding below zero; NaN stays NaN
+            a.ent_out[r] = H;
+            a.tok_out[r] = (t.bi == INT_MAX || t.bi < 0 || t.bi >= a.V) ? 0 : t.bi;
+            if (H != H) atomicAdd(&a.stat->nan_rows, 1u);
+        }
+    }
+}
+
+// Eq. 2 / Algorithm 1: mask = H > tau (strict); a NaN entropy routes to the LLM.
+__device__ __forceinline__ uint8_t rule(float H, float tau)
+{
+    return (H != H || H > tau) ? 1 : 0;
+}
+
+// S4: per-sequence mask from per-row entropies already in global memory (written by this block).
+__device__ inline void tail_mask(const TailArgs &a)
+{
+    if (a.row_seq == nullptr) {
+        for (int b = threadIdx.x; b < a.B; b += blockDim.x)
+            a.route_mask[b] = (b < a.R) ? rule(a.ent_out[b], a.tau) : 0;
+    } else {
+        for (int b = threadIdx.x; b < a.B; b += blockDim.x) a.route_mask[b] = 0;
+        __syncthreads();
+        for (int r = threadIdx.x; r < a.R; r += blockDim.x) {
+            int sq = a.row_seq[r];
+            bool last = (r == a.R - 1) || (a.row_seq[r + 1] != sq);
+            if (last && sq >= 0 && sq < a.B) a.route_mask[sq] = rule(a.ent_out[r], a.tau);
+        }
+    }
+    __syncthreads();
+}
+
+// S5 + S6 by one block: chunks of blockDim.x sequences; inside a chunk a warp ballot gives each
+// routed sequence its rank in the warp, per-warp totals are scanned in shared memory, and a
+// running carry links the chunks, so llm_idx comes out ascending.  Spans get the same treatment
+// with an inclusive warp scan.  smem: at least 2 * 32 + 2 ints.
+__device__ inline void tail_compact(const uint8_t *mask, int B, const int32_t *seq_len,
+                                    const int32_t *kv_len, int32_t *llm_idx, int32_t *llm_count,
+                                    int32_t *llm_span, int32_t *llm_row_off, DevStat *stat,
+                                    int *smem /* >= 66 ints */)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    int *w_cnt = smem, *w_rows = smem + 32, *carry = smem + 64;     // carry[0] = count, carry[1] = rows
+    if (threadIdx.x == 0) { carry[0] = 0; carry[1] = 0; }
+    __syncthreads();
+    const bool spans = (seq_len != nullptr);
+    for (int base = 0; base < B; base += blockDim.x) {
+        int b = base + threadIdx.x;
+        bool routed = (b < B) && (mask[b] != 0);
+        unsigned ball = __ballot_sync(0xffffffffu, routed);
+        int rank = __popc(ball & ((1u << lane) - 1u));
+        int span = 0, incl = 0;
+        if (spans) {
+            if (routed) {
+                span = seq_len[b] - kv_len[b];
+                if (span < 1) atomicAdd(&stat->bad_span, 1u);
+            }
+            incl = span;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+        }
+        if (lane == 31) { w_cnt[warp] = __popc(ball); w_rows[warp] = incl; }
+        __syncthreads();
+        int pre_cnt = carry[0], pre_rows = carry[1];
+        for (int w = 0; w < warp; ++w) { pre_cnt += w_cnt[w]; pre_rows += w_rows[w]; }
+        if (routed) {
+            int j = pre_cnt + rank;
+            llm_idx[j] = b;
+            if (spans) { llm_span[j] = span; llm_row_off[j] = pre_rows + incl - span; }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int c = 0, rws = 0;
+            for (int w = 0; w < nwarps; ++w) { c += w_cnt[w]; rws += w_rows[w]; }
+            carry[0] += c; carry[1] += rws;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        *llm_count = carry[0];
+        if (spans) llm_row_off[carry[0]] = carry[1];
+    }
+}
+
+__device__ inline void tail_route(const TailArgs &a, int *smem)
+{
+    tail_mask(a);
+    tail_compact(a.route_mask, a.B, a.seq_len, a.kv_len, a.llm_idx, a.llm_count, a.llm_span,
+                 a.llm_row_off, a.stat, smem);
+}
+
+}  // namespace rstitch

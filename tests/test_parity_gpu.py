@@ -1,0 +1,262 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same
+seeded bf16 inputs (element by element at sizes the oracle finishes in seconds)."""
+import math
+
+import numpy as np
+import pytest
+
+import rstitch_inputs as gen
+from parity_util import compare, run_gpu, to_dev_bf16, to_dev_i32
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rs():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2507_17307_b200 import build
+    build.build_library()
+    import paper_2507_17307_b200 as rs
+    return rs
+
+
+@pytest.fixture(scope="module")
+def handle(rs):
+    h = rs.Handle(1024, 8192, 160000)
+    yield h
+    h.destroy()
+
+
+def check_case(rs, handle, oracle, w, steps, tau=None, flags=0, w_bits=None, w_dev=None):
+    tau = w.tau_nats if tau is None else tau
+    if w_bits is None:
+        w_bits = gen.make_w_head(w)
+    if w_dev is None:
+        w_dev = to_dev_bf16(w_bits)
+    stats = []
+    for step in steps:
+        hid, _ = gen.make_hidden(w, w_bits, step)
+        seq_len, kv_len = gen.make_kv_state(w, step)
+        ref = oracle.route(hid, w_bits, tau, seq_len=seq_len, kv_len=kv_len)
+        gpu = run_gpu(handle, hid, w_dev, tau, seq_len=seq_len, kv_len=kv_len, flags=flags)
+        stats.append(compare(gpu, ref, tau, w.B, w.B, oracle=oracle, seq_len=seq_len, kv_len=kv_len))
+    st = rs.last_status(handle)
+    assert st["status"] == 0 and st["nan_rows"] == 0 and st["bad_span"] == 0 and st["timeouts"] == 0
+    return stats
+
+
+def test_c1_tiny_all_steps(rs, handle, oracle):
+    w = gen.WORKLOADS["c1_tiny"]
+    stats = check_case(rs, handle, oracle, w, range(w.steps))
+    assert max(s["max_ent_err"] for s in stats) < 1e-3
+
+
+@pytest.mark.parametrize("B", [1, 2, 3, 4, 5, 7, 16, 17])
+@pytest.mark.parametrize("d,V", [(8, 2), (8, 3), (64, 1000), (256, 4097), (1536, 2053), (24, 777)])
+def test_shapes_and_ragged_tails(rs, handle, oracle, B, d, V):
+    w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=d, V=V, seed=7000 + B + d + V,
+                   sigma_w=0.5 / math.sqrt(d))
+    check_case(rs, handle, oracle, w, [0, 1])
+
+
+@pytest.mark.parametrize("name,V,B", [("c2_slm_b1", 9001, 1), ("c3_llm_b1", 6007, 1), ("c3_llm_b4", 6007, 4),
+                                       ("c3_llm_b16", 6007, 16), ("c4_slm_b64", 5003, 64),
+                                       ("c4_llm_b64", 3001, 23)])
+def test_reduced_vocab_workloads(rs, handle, oracle, name, V, B):
+    # the paper-shaped heads with the vocabulary cut down so that the oracle covers every row
+    w = gen.scaled(gen.WORKLOADS[name], V=V, B=B)
+    stats = check_case(rs, handle, oracle, w, [0, 1, 2])
+    if name.startswith(("c3", "c4")):
+        rates = [s["route_rate"] for s in stats]
+        assert 0.0 <= min(rates) and max(rates) <= 1.0
+
+
+def test_all_routed_none_routed_and_threshold_ends(rs, handle, oracle):
+    w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], V=2048, d=128, B=64, sigma_w=0.05)
+    w_bits = gen.make_w_head(w)
+    w_dev = to_dev_bf16(w_bits)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    for tau, expect in [(-1.0, 64), (100.0, 0)]:
+        ref = oracle.route(hid, w_bits, tau)
+        gpu = run_gpu(handle, hid, w_dev, tau)
+        compare(gpu, ref, tau, 64, 64)
+        assert int(gpu["llm_count"][0]) == expect
+    # exactly one routed sequence, at either end: threshold between the largest entropies
+    ref = oracle.route(hid, w_bits, 0.0)
+    order = np.argsort(ref["ent"])
+    tau = 0.5 * (ref["ent"][order[-1]] + ref["ent"][order[-2]])
+    if ref["ent"][order[-1]] - ref["ent"][order[-2]] > 0.01:
+        gpu = run_gpu(handle, hid, w_dev, tau)
+        assert int(gpu["llm_count"][0]) == 1 and gpu["llm_idx"][0] == order[-1]
+
+
+def test_normalized_tau_flag(rs, handle, oracle):
+    w = gen.scaled(gen.WORKLOADS["c3_llm_b16"], V=4096, d=256)
+    w_bits = gen.make_w_head(w)
+    hid, _ = gen.make_hidden(w, w_bits, 5)
+    for tau_paper in (0.0005, 0.001, 0.005, 0.01, 0.02, 0.03, 0.05):
+        tau_nats = tau_paper * math.log(w.V)
+        ref = oracle.route(hid, w_bits, tau_nats)
+        gpu = run_gpu(handle, hid, to_dev_bf16(w_bits), tau_paper, flags=rs.TAU_NORMALIZED)
+        compare(gpu, ref, tau_nats, w.B, w.B)
+
+
+def test_row_gather_and_live_row_count(rs, handle, oracle):
+    # the LLM head on the compacted subset of an earlier call: row_idx = llm_idx, rows = llm_count
+    w = gen.scaled(gen.WORKLOADS["c4_llm_b64"], V=3000, d=512, B=64)
+    w_bits = gen.make_w_head(w)
+    w_dev = to_dev_bf16(w_bits)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    row_idx = np.array([3, 9, 10, 31, 40, 63, 0, 0], dtype=np.int32)
+    live = 6
+    ref = oracle.route(hid, w_bits, w.tau_nats, row_idx=row_idx[:live])
+    gpu = run_gpu(handle, hid, w_dev, w.tau_nats, row_idx=row_idx, n_rows_dev=live, R=8)
+    compare(gpu, ref, w.tau_nats, live, live)
+    assert (gpu["tok"][live:8] == -1).all() and (gpu["ent"][live:8] == -1.0).all()
+    assert (gpu["mask"][live:8] == 255).all()
+    # an out-of-range gather entry is counted, not dereferenced
+    bad = np.array([1, 64, -5, 2], dtype=np.int32)
+    gpu = run_gpu(handle, hid, w_dev, w.tau_nats, row_idx=bad)
+    ref = oracle.route(hid, w_bits, w.tau_nats, row_idx=np.array([1, 0, 0, 2], dtype=np.int32))
+    compare(gpu, ref, w.tau_nats, 4, 4)
+    assert rs.last_status(handle)["bad_row_idx"] == 2
+
+
+def test_multi_row_spans_decide_on_last_row(rs, handle, oracle):
+    w = gen.scaled(gen.WORKLOADS["c5_catchup"], V=2500, d=320, B=12)
+    w_bits = gen.make_w_head(w)
+    k = gen.make_spans(w, 0)
+    R = int(k.sum())
+    row_seq = np.repeat(np.arange(w.B, dtype=np.int32), k)
+    hid, _ = gen.make_hidden(w, w_bits, 0, rows=R)
+    seq_len, kv_len = gen.make_kv_state(w, 0, span=k)
+    ref = oracle.route(hid, w_bits, w.tau_nats, row_seq=row_seq, B=w.B, seq_len=seq_len, kv_len=kv_len)
+    gpu = run_gpu(handle, hid, to_dev_bf16(w_bits), w.tau_nats, row_seq=row_seq, B=w.B,
+                  seq_len=seq_len, kv_len=kv_len)
+    compare(gpu, ref, w.tau_nats, R, w.B, row_seq=row_seq, oracle=oracle, seq_len=seq_len, kv_len=kv_len)
+    cnt = int(gpu["llm_count"][0])
+    assert gpu["llm_row_off"][cnt] == k[gpu["llm_idx"][:cnt]].sum()
+
+
+def test_bad_span_is_counted(rs, handle, oracle):
+    w = gen.scaled(gen.WORKLOADS["c1_tiny"], V=512, d=64, B=4)
+    w_bits = gen.make_w_head(w)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    seq_len = np.array([10, 10, 10, 10], dtype=np.int32)
+    kv_len = np.array([9, 10, 12, 5], dtype=np.int32)
+    gpu = run_gpu(handle, hid, to_dev_bf16(w_bits), -1.0, seq_len=seq_len, kv_len=kv_len)
+    assert gpu["llm_span"][:4].tolist() == [1, 0, -2, 5]
+    assert rs.last_status(handle)["bad_span"] == 2
+
+
+def test_nan_row_is_routed_and_counted(rs, handle, oracle):
+    w = gen.scaled(gen.WORKLOADS["c1_tiny"], V=1024, d=64, B=3)
+    w_bits = gen.make_w_head(w)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    hid[1, 5] = 0x7FC0
+    ref = oracle.route(hid, w_bits, 100.0)
+    gpu = run_gpu(handle, hid, to_dev_bf16(w_bits), 100.0)
+    compare(gpu, ref, 100.0, 3, 3)
+    assert gpu["mask"][:3].tolist() == [0, 1, 0] and gpu["tok"][1] == 0
+    assert rs.last_status(handle)["nan_rows"] == 1
+
+
+def test_determinism_bitwise(rs, handle):
+    w = gen.scaled(gen.WORKLOADS["c3_llm_b16"], V=20011, d=512)
+    w_bits = gen.make_w_head(w)
+    w_dev = to_dev_bf16(w_bits)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    a = run_gpu(handle, hid, w_dev, w.tau_nats)
+    for _ in range(3):
+        b = run_gpu(handle, hid, w_dev, w.tau_nats)
+        for k in a:
+            assert np.array_equal(a[k].view(np.uint8), b[k].view(np.uint8)), k
+
+
+def test_basic_entry_point_and_empty_batch(rs, oracle):
+    import torch
+    w = gen.WORKLOADS["c1_tiny"]
+    w_bits = gen.make_w_head(w)
+    hid, _ = gen.make_hidden(w, w_bits, 1)
+    out = rs.route(to_dev_bf16(hid), to_dev_bf16(w_bits), w.tau_nats)
+    torch.cuda.synchronize()
+    ref = oracle.route(hid, w_bits, w.tau_nats)
+    gpu = {k: getattr(out, k).cpu().numpy() for k in ("tok", "ent", "mask", "llm_idx", "llm_count")}
+    compare(gpu, ref, w.tau_nats, w.B, w.B)
+    # B = 0: valid, count = 0, nothing else touched
+    empty = torch.empty((0, w.d), dtype=torch.bfloat16, device="cuda")
+    out = rs.route(empty, to_dev_bf16(w_bits), w.tau_nats)
+    torch.cuda.synchronize()
+    assert int(out.llm_count.item()) == 0 and int(out.tok[0].item()) == -1
+
+
+def test_host_buffer_entry_point(rs, handle, oracle):
+    import torch
+    w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], V=4099, d=256, B=64)
+    w_bits = gen.make_w_head(w)
+    hid, _ = gen.make_hidden(w, w_bits, 2)
+    hh = torch.from_numpy(hid.view(np.int16)).view(torch.bfloat16).pin_memory()
+    host = {"tok": torch.full((64,), -1, dtype=torch.int32).pin_memory(),
+            "ent": torch.zeros(64, dtype=torch.float32).pin_memory(),
+            "mask": torch.zeros(64, dtype=torch.uint8).pin_memory(),
+            "llm_idx": torch.full((64,), -1, dtype=torch.int32).pin_memory(),
+            "llm_count": torch.zeros(1, dtype=torch.int32).pin_memory()}
+    rs.route_host(handle, hh, to_dev_bf16(w_bits), w.tau_nats, host)
+    ref = oracle.route(hid, w_bits, w.tau_nats)
+    gpu = {k: v.numpy() for k, v in host.items()}
+    cnt = int(gpu["llm_count"][0])
+    gpu["llm_idx"][cnt:] = -1          # the copy brings back the whole staging array
+    compare(gpu, ref, w.tau_nats, 64, 64)
+
+
+def test_caller_workspace(rs, handle, oracle):
+    import torch
+    w = gen.scaled(gen.WORKLOADS["c3_llm_b4"], V=3001, d=128)
+    w_bits = gen.make_w_head(w)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    n = rs.workspace_bytes(w.B, w.d, w.V)
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda").fill_(0xAB)
+    out = rs.route_ex(handle, to_dev_bf16(hid), to_dev_bf16(w_bits), w.tau_nats, workspace=ws)
+    torch.cuda.synchronize()
+    ref = oracle.route(hid, w_bits, w.tau_nats)
+    gpu = {k: getattr(out, k).cpu().numpy() for k in ("tok", "ent", "mask", "llm_idx", "llm_count")}
+    compare(gpu, ref, w.tau_nats, w.B, w.B)
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    assert rs.route_ex(handle, to_dev_bf16(hid), to_dev_bf16(w_bits), 0.3, workspace=small, check=False) == -5
+
+
+def test_device_side_argument_errors(rs, handle):
+    import torch
+    w_dev = torch.zeros((64, 32), dtype=torch.bfloat16, device="cuda")
+    hid = torch.zeros((5, 32), dtype=torch.bfloat16, device="cuda")
+    assert rs.route_ex(handle, hid, w_dev, float("nan"), check=False) == -1
+    assert rs.route_ex(handle, hid, w_dev, 0.3, B=3, check=False) == -1          # B != R without row_seq
+    assert rs.route_ex(handle, hid, w_dev, 0.3, flags=0x30, check=False) == -1
+    assert rs.route_ex(handle, hid, w_dev, 0.3, flags=0x4000, check=False) == -1         # unknown flag
+    flat = torch.zeros(5 * 32 + 8, dtype=torch.bfloat16, device="cuda")
+    mis = flat[1:1 + 5 * 32].view(5, 32)                                           # 2-byte offset
+    assert rs.route_ex(handle, mis, w_dev, 0.3, check=False) == -2
+    big = torch.zeros((2, 16384 + 8), dtype=torch.bfloat16, device="cuda")
+    wbig = torch.zeros((4, 16384 + 8), dtype=torch.bfloat16, device="cuda")
+    assert rs.route_ex(handle, big, wbig, 0.3, check=False) == -3
+
+
+@pytest.mark.parametrize("B", [0, 1, 31, 32, 33, 255, 256, 257, 1000, 65536, 65537, 300001])
+def test_standalone_compaction(rs, oracle, B):
+    import torch
+    for p in (0.1, 0.5, 0.9):
+        m = gen.random_mask(B, p, seed=B)
+        md = torch.from_numpy(m).cuda() if B else torch.zeros(0, dtype=torch.uint8, device="cuda")
+        idx, cnt = rs.compact(md)
+        torch.cuda.synchronize()
+        ref_idx, ref_cnt = oracle.compact(m)
+        assert int(cnt.item()) == ref_cnt
+        assert np.array_equal(idx.cpu().numpy()[:ref_cnt], ref_idx)
+        if B:
+            assert (idx.cpu().numpy()[ref_cnt:] == -1).all()
+    for fill in (0, 1):
+        if B:
+            md = torch.full((B,), fill, dtype=torch.uint8, device="cuda")
+            idx, cnt = rs.compact(md)
+            assert int(cnt.item()) == fill * B
