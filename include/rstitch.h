@@ -150,6 +150,32 @@ int rstitch_route_host(rstitch_handle_t h, const void *hidden_host, const void *
                        int32_t *tok_host, float *ent_host, uint8_t *mask_host,
                        int32_t *llm_idx_host, int32_t *llm_count_host, void *cuda_stream);
 
+/*
+ * The same decision as rstitch_route (S1-S5, B rows, one decision per row) for callers that cannot
+ * allocate device memory.  (The paper has no counterpart; this is a deployment variant.)
+ *
+ * Who needs it: code running inside a serving engine whose memory pool already owns the whole
+ * device, a decode loop that cannot afford the device-wide synchronisation an allocation may cause,
+ * or a process whose device budget is fixed at start-up.  This entry point calls no cudaMalloc,
+ * cudaFree or any other allocating routine, on any call: its scratch (ticket counter, per-slice
+ * partial statistics, status word) is a fixed array of about RSTITCH_STATIC_MAX_ROWS * 20 KiB inside
+ * the library image, which every GPU that loads the library holds until the process exits.
+ *
+ *  - B > RSTITCH_STATIC_MAX_ROWS returns RSTITCH_ERR_UNSUPPORTED_SHAPE (the scratch is fixed); the
+ *    other argument rules are those of rstitch_route.  Inputs and outputs are still the caller's.
+ *  - The first call on each device looks up the array's device address (no allocation); make that
+ *    first call with the device current and before any stream capture begins.
+ *  - All calls on a device share the one array, which keeps the previous call's contents: each call
+ *    clears what must start at zero on the given stream.  Two calls that overlap on the GPU (different
+ *    streams, no ordering between them) race on it; order them.
+ *  - No status word is reported back: NaN rows are still routed, but not counted anywhere.
+ */
+#define RSTITCH_STATIC_MAX_ROWS 16
+int rstitch_route_static(const void *hidden /* bf16 [B,d] */, const void *W_head /* bf16 [V,d] */,
+                         int B, int d, int V, float tau /* nats */,
+                         int32_t *tok_out, float *ent_out, uint8_t *route_mask, int32_t *llm_idx,
+                         int32_t *llm_count, void *cuda_stream);
+
 /* Handle: owns the scratch memory and the device status word for problems up to the given maxima on
  * the current device.  rstitch_destroy(NULL) is a no-op. */
 int rstitch_create(rstitch_handle_t *out, int maxR, int max_d, int maxV);

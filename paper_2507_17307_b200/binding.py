@@ -20,7 +20,7 @@ PATH_UMMA = 0x20
 EXPORTS = [
     "rstitch_route", "rstitch_route_ex", "rstitch_route_host", "rstitch_create", "rstitch_destroy",
     "rstitch_workspace_bytes", "rstitch_compact", "rstitch_last_status", "rstitch_status_string",
-    "rstitch_path_name",
+    "rstitch_path_name", "rstitch_route_static",
 ]
 
 
@@ -88,6 +88,8 @@ def lib():
         L.rstitch_status_string.restype = C.c_char_p
         L.rstitch_path_name.argtypes = [i, i, i, C.c_uint32]
         L.rstitch_path_name.restype = C.c_char_p
+        L.rstitch_route_static.argtypes = [vp, vp, i, i, i, f, vp, vp, vp, vp, vp, vp]
+        L.rstitch_route_static.restype = i
         _lib = L
     return _lib
 
@@ -210,6 +212,24 @@ def route_ex(handle: Handle, hidden, W_head, tau: float, *, R: Optional[int] = N
     if st != 0:
         raise RstitchError(st, "rstitch_route_ex")
     return out
+
+
+STATIC_MAX_ROWS = 16
+
+
+def route_static(hidden, W_head, tau: float, out: RouteOutputs, stream=None, check: bool = True):
+    """rstitch_route_static: the allocation-free variant (scratch inside the library image).
+
+    For callers that may not allocate device memory, so `out` must be given: this wrapper creates
+    no tensor.  At most STATIC_MAX_ROWS rows; calls sharing a device must not overlap on the GPU.
+    """
+    B, d = int(hidden.shape[0]), int(hidden.shape[1])
+    st = lib().rstitch_route_static(_ptr(hidden), _ptr(W_head), B, d, int(W_head.shape[0]), float(tau),
+                                    _ptr(out.tok), _ptr(out.ent), _ptr(out.mask), _ptr(out.llm_idx),
+                                    _ptr(out.llm_count), _stream_ptr(stream))
+    if check and st != 0:
+        raise RstitchError(st, "rstitch_route_static")
+    return out if check else st
 
 
 class PreparedCall:
