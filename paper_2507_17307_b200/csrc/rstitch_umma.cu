@@ -1,0 +1,485 @@
+// Tensor-core LM-head kernel (S1-S3 fused): hidden rows on the M side of tcgen05.mma, vocabulary
+// on the N side, fp32 accumulators in tensor memory, and an epilogue that turns each accumulator
+// tile into single-pass softmax statistics and the greedy token without the logits ever leaving
+// the SM.
+//
+// Block = 6 warps, one block per SM:
+//   warp 0  producer: one thread issues tensor-map (TMA) copies of a 128 x 64 hidden tile and an
+//           N x 64 W_head tile (128-byte swizzle) into a 4-stage shared-memory ring;
+//   warp 1  one thread issues the tcgen05.mma instructions (M = 128, N <= 256, K = 16) and commits
+//           them to the ring's "empty" barriers and to the accumulator's "full" barrier; the warp
+//           also owns the tensor-memory allocation (512 columns = two 256-column accumulators);
+//   warps 2-5  epilogue: thread = one hidden row (one TMEM lane); it reads its row of the
+//           accumulator 32 columns at a time and folds the logits into (m, s, u, argmax).
+// The two accumulators alternate, so the epilogue of one tile runs under the MMAs of the next.
+//
+// Work split.  Up to 128 rows (one M tile): each block owns one contiguous, balanced range of the
+// vocabulary, cut into tiles of at most 256 rows, and keeps one running statistic per row; W_head
+// is read from HBM exactly once and the kernel is HBM-bound.  More rows: work items are
+// (256-row vocabulary tile, 128-row M tile) pairs dealt round-robin with the M tiles of one
+// vocabulary tile adjacent, so that they run at the same time on neighbouring SMs and W_head
+// comes from HBM once and from L2 for the other M tiles.
+#include "rstitch_kernels.cuh"
+#include "rstitch_ptx.cuh"
+
+#include <cuda.h>
+
+namespace rstitch {
+
+namespace {
+
+constexpr int kThreads   = 192;
+constexpr int kStages    = 4;
+constexpr int kTileM     = 128;
+constexpr int kTileNMax  = 256;
+constexpr int kTileK     = 64;                       // bf16 elements = one 128-byte swizzle row
+constexpr int kABytes    = kTileM * kTileK * 2;      // 16 KB
+constexpr int kBBytes    = kTileNMax * kTileK * 2;   // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kDynSmem   = kStages * kStageBytes + 1024;   // + slack to align the ring to 1024 B
+constexpr int kTmemCols  = 512;
+
+struct Item { int v0, N, m; };
+
+// The work item a block takes at its j-th iteration; identical in every role of the block.
+struct Schedule {
+    int V, nM, grid, cta;
+    // one M tile: balanced contiguous ranges in units of 16 vocabulary rows
+    int u_begin, nu, n_tiles;
+    // several M tiles
+    int n_items;
+
+    __device__ void init(int V_, int nM_, int grid_, int cta_)
+    {
+        V = V_; nM = nM_; grid = grid_; cta = cta_;
+        if (nM == 1) {
+            long long units = (V + 15) / 16;
+            u_begin = (int)(units * cta / grid);
+            int u_end = (int)(units * (cta + 1) / grid);
+            nu = u_end - u_begin;
+            n_tiles = (nu + 15) / 16;
+            n_items = n_tiles;
+        } else {
+            int nVT = (V + kTileNMax - 1) / kTileNMax;
+            int total = nVT * nM;
+            n_items = cta < total ? (total - cta + grid - 1) / grid : 0;
+        }
+    }
+    __device__ Item item(int j) const
+    {
+        Item it;
+        if (nM == 1) {
+            int a = u_begin + (int)((long long)nu * j / n_tiles);
+            int b = u_begin + (int)((long long)nu * (j + 1) / n_tiles);
+            it.v0 = a * 16; it.N = (b - a) * 16; it.m = 0;
+        } else {
+            int q = cta + j * grid;
+            int vt = q / nM;
+            it.m = q - vt * nM;
+            it.v0 = vt * kTileNMax;
+            int left = V - it.v0;
+            it.N = left >= kTileNMax ? kTileNMax : ((left + 15) / 16) * 16;
+        }
+        return it;
+    }
+};
+
+__device__ __forceinline__ void raise_abort(volatile int *flag, DevStat *stat, unsigned site)
+{
+    *flag = 1;
+    atomicAdd(&stat->timeouts, 1u);
+    atomicExch(&stat->timeout_site, site);
+}
+
+// Fold up to 32 logits (columns c0 .. c0+31 of the tile, vocabulary index v0 + column) into the
+// row's statistics.  n_valid = how many of them are real vocabulary entries.
+__device__ __forceinline__ void fold_chunk(Stats &st, const float (&z)[32], int n_valid, int vbase)
+{
+    float cmax = -CUDART_INF_F;
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (i < n_valid) cmax = fmaxf(cmax, z[i]);
+    const float m_new = fmaxf(st.m, cmax);
+    if (st.m == -CUDART_INF_F) { st.s = 0.f; st.u = 0.f; }
+    else {
+        float dm = st.m - m_new;
+        float a = __expf(dm);
+        st.u = a * (st.u + dm * st.s);
+        st.s = a * st.s;
+    }
+    st.m = m_new;
+    float s = 0.f, u = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        if (i < n_valid) {
+            float dz = z[i] - m_new;
+            float e = __expf(dz);
+            s += e;
+            u = fmaf(e, dz, u);
+            if (z[i] > st.bv) { st.bv = z[i]; st.bi = vbase + i; }   // ascending index: first maximum wins
+        }
+    }
+    st.s += s;
+    st.u += u;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_constant__ CUtensorMap tm_w32,
+                 const __grid_constant__ CUtensorMap tm_w16, const __grid_constant__ CUtensorMap tm_w256,
+                 HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int nM, int n_slices)
+{
+    extern __shared__ unsigned char dyn_smem_raw[];
+    __shared__ __align__(8) uint64_t s_full[kStages], s_empty[kStages];
+    __shared__ __align__(8) uint64_t s_acc_full[2], s_acc_empty[2], s_done;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_tail[66];
+    __shared__ int s_last, s_abort, s_zero;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ring = (ptx::smem_u32(dyn_smem_raw) + 1023u) & ~1023u;
+    const int nK = (h.d + kTileK - 1) / kTileK;
+    int R_live = h.R;
+    if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
+
+    Schedule sch;
+    sch.init(h.V, nM, gridDim.x, blockIdx.x);
+
+    if (threadIdx.x == 0) {
+        s_abort = 0; s_zero = 0;
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&s_full[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&s_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(ptx::smem_u32(&s_acc_full[b]), 1);
+            ptx::mbar_init(ptx::smem_u32(&s_acc_empty[b]), 4);     // one arrival per epilogue warp
+        }
+        ptx::mbar_init(ptx::smem_u32(&s_done), 1);
+        ptx::mbar_fence_init();
+        ptx::prefetch_tmap(&tm_hidden);
+        ptx::prefetch_tmap(nM == 1 ? &tm_w32 : &tm_w256);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(&s_tmem_base), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = s_tmem_base;
+
+    if (warp == 0) {
+        // ---- producer --------------------------------------------------------------------
+        if (lane == 0) {
+            int stage = 0, round = 0, issued = 0;
+            bool live = true;
+            for (int j = 0; live && j < sch.n_items; ++j) {
+                const Item it = sch.item(j);
+                for (int ks = 0; ks < nK; ++ks) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&s_empty[stage]), (uint32_t)((round & 1) ^ 1), &s_abort)) {
+                        if (!s_abort) raise_abort(&s_abort, t.stat, 0x201u);
+                        live = false;
+                        break;
+                    }
+                    const uint32_t full = ptx::smem_u32(&s_full[stage]);
+                    const uint32_t a_dst = ring + (uint32_t)stage * kStageBytes;
+                    const uint32_t b_dst = a_dst + kABytes;
+                    ptx::mbar_arrive_expect_tx(full, (uint32_t)(kABytes + it.N * kTileK * 2));
+                    ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, it.m * kTileM, full);
+                    if (it.N == kTileNMax) {
+                        ptx::tma_g2s_2d(b_dst, &tm_w256, ks * kTileK, it.v0, full);
+                    } else {
+                        int r = 0;
+                        for (; r + 32 <= it.N; r += 32)
+                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w32, ks * kTileK, it.v0 + r, full);
+                        if (r < it.N)
+                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w16, ks * kTileK, it.v0 + r, full);
+                    }
+                    ++issued;
+                    if (++stage == kStages) { stage = 0; ++round; }
+                }
+            }
+            if (s_abort) {
+                // no copy may still be landing in this block's shared memory when it exits
+                int first = issued > kStages ? issued - kStages : 0;
+                for (int q = first; q < issued; ++q)
+                    ptx::mbar_wait(ptx::smem_u32(&s_full[q % kStages]), (uint32_t)((q / kStages) & 1), &s_zero);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---- MMA issuer ------------------------------------------------------------------
+        if (lane == 0) {
+            int stage = 0, round = 0;
+            bool live = true;
+            for (int j = 0; live && j < sch.n_items; ++j) {
+                const Item it = sch.item(j);
+                const int buf = j & 1, use = j >> 1;
+                if (!ptx::mbar_wait(ptx::smem_u32(&s_acc_empty[buf]), (uint32_t)((use & 1) ^ 1), &s_abort)) {
+                    if (!s_abort) raise_abort(&s_abort, t.stat, 0x202u);
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, it.N);
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kTileNMax;
+                for (int ks = 0; ks < nK; ++ks) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&s_full[stage]), (uint32_t)(round & 1), &s_abort)) {
+                        if (!s_abort) raise_abort(&s_abort, t.stat, 0x203u);
+                        live = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_src = ring + (uint32_t)stage * kStageBytes;
+                    const uint64_t a_desc = ptx::smem_desc_sw128(a_src);
+                    const uint64_t b_desc = ptx::smem_desc_sw128(a_src + kABytes);
+#pragma unroll
+                    for (int kk = 0; kk < kTileK / 16; ++kk)     // 32 bytes along K per instruction
+                        ptx::umma_bf16(d_tmem, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc,
+                                       (uint32_t)((ks | kk) != 0));
+                    ptx::umma_commit(ptx::smem_u32(&s_empty[stage]));      // frees the stage when the MMAs are done
+                    if (++stage == kStages) { stage = 0; ++round; }
+                }
+                if (live) ptx::umma_commit(ptx::smem_u32(&s_acc_full[buf]));   // accumulator complete
+            }
+            // everything issued has finished before the tensor memory is released
+            ptx::umma_commit(ptx::smem_u32(&s_done));
+            ptx::mbar_wait(ptx::smem_u32(&s_done), 0u, &s_zero);
+        }
+        __syncwarp();
+    } else {
+        // ---- epilogue --------------------------------------------------------------------
+        const int quarter = warp & 3;                        // the TMEM lanes this warp may read
+        const int row_in_tile = quarter * 32 + lane;
+        Stats st = stats_empty();
+        for (int j = 0; j < sch.n_items; ++j) {
+            const Item it = sch.item(j);
+            const int buf = j & 1, use = j >> 1;
+            const int row = it.m * kTileM + row_in_tile;
+            if (!ptx::mbar_wait(ptx::smem_u32(&s_acc_full[buf]), (uint32_t)(use & 1), &s_abort)) {
+                if (lane == 0 && !s_abort) raise_abort(&s_abort, t.stat, 0x204u);
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            const bool warp_has_rows = (it.m * kTileM + quarter * 32) < R_live;
+            if (nM > 1) st = stats_empty();
+            if (warp_has_rows) {
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kTileNMax;
+                for (int c0 = 0; c0 < it.N; c0 += 32) {
+                    float z[32];
+                    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, z);
+                    int n_valid = it.N - c0;
+                    if (h.V - (it.v0 + c0) < n_valid) n_valid = h.V - (it.v0 + c0);
+                    if (n_valid > 32) n_valid = 32;
+                    if (row < R_live && n_valid > 0) fold_chunk(st, z, n_valid, it.v0 + c0);
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&s_acc_empty[buf]));
+            if (nM > 1 && row < R_live)
+                partial_store(P, (size_t)row * n_slices + (size_t)(it.v0 / kTileNMax), st);
+        }
+        if (nM == 1 && row_in_tile < R_live)
+            partial_store(P, (size_t)row_in_tile * n_slices + blockIdx.x, st);
+    }
+
+    ptx::tc_fence_before_sync();
+    __threadfence();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (nM > 1) return;               // several M tiles: a separate kernel merges the partials
+
+    // one M tile: the last block done merges all slices and runs the routing tail
+    if (threadIdx.x == 0) {
+        unsigned k = atomicAdd(ticket, 1u);
+        s_last = (k == (unsigned)(gridDim.x - 1));
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    TailArgs ta = t;
+    ta.R = R_live;
+    if (h.n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
+    tail_finalize_rows(P, n_slices, ta);
+    __syncthreads();
+    tail_route(ta, s_tail);
+    if (threadIdx.x == 0) {
+        *ticket = 0u;
+        atomicAdd(&t.stat->launches, 1u);
+    }
+}
+
+// Several M tiles: one warp per row merges that row's per-tile partials; the last block done
+// applies the rule and compacts.
+__global__ void __launch_bounds__(256)
+head_finalize_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_slices)
+{
+    __shared__ int s_tail[66];
+    __shared__ int s_last;
+    int R_live = h.R;
+    if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (r < R_live) {
+        Stats st = stats_empty();
+        for (int c = lane; c < n_slices; c += 32) {
+            Stats p = partial_load(P, (size_t)r * n_slices + c);
+            stats_merge(st, p);
+        }
+        stats_warp_allmerge(st);
+        if (lane == 0) {
+            float H = logf(st.s) - st.u / st.s;
+            if (H < 0.f) H = 0.f;
+            t.ent_out[r] = H;
+            t.tok_out[r] = (st.bi == INT_MAX || st.bi < 0 || st.bi >= t.V) ? 0 : st.bi;
+            if (H != H) atomicAdd(&t.stat->nan_rows, 1u);
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned k = atomicAdd(ticket, 1u);
+        s_last = (k == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    TailArgs ta = t;
+    ta.R = R_live;
+    if (h.n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
+    tail_route(ta, s_tail);
+    if (threadIdx.x == 0) {
+        *ticket = 0u;
+        atomicAdd(&t.stat->launches, 1u);
+    }
+}
+
+// hidden[row_idx[r]] -> packed[r] (zero for rows past the live count or with a bad index).
+__global__ void __launch_bounds__(128)
+gather_rows_kernel(HeadArgs h, uint4 *packed, int rows_padded, DevStat *stat)
+{
+    const int r = blockIdx.x;
+    const int d8 = h.d >> 3;
+    int R_live = h.R;
+    if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
+    int src = -1;
+    if (r < R_live) {
+        src = h.row_idx ? h.row_idx[r] : r;
+        if (src < 0 || src >= h.n_src) {
+            if (threadIdx.x == 0) atomicAdd(&stat->bad_row_idx, 1u);
+            src = 0;
+        }
+    }
+    const uint4 *in = (const uint4 *)h.hidden;
+    for (int c = threadIdx.x; c < d8; c += blockDim.x)
+        packed[(size_t)r * d8 + c] = src >= 0 ? in[(size_t)src * d8 + c] : make_uint4(0, 0, 0, 0);
+    (void)rows_padded;
+}
+
+// ---- host side: tensor maps -----------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// bf16 [rows, d] row-major, box = 64 elements along d by box_rows rows, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool make_map(CUtensorMap *m, const void *base, int rows, int d, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2]    = {(cuuint64_t)d, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+    cuuint32_t box[2]     = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2]    = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool umma_shape_ok(int R, int d, int V)
+{
+    return R >= 1 && d >= kTileK && V >= kTileNMax && encode_fn() != nullptr;
+}
+
+int umma_slices(int R, int V, int sm_count)
+{
+    return R <= kTileM ? sm_count : (V + kTileNMax - 1) / kTileNMax;
+}
+
+size_t umma_gather_bytes(int R, int d)
+{
+    size_t rows = (size_t)((R + kTileM - 1) / kTileM) * kTileM;
+    return rows * (size_t)d * 2;
+}
+
+cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
+                             int sm_count, cudaStream_t stream)
+{
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        e = cudaFuncSetAttribute(head_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmem);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    const int nM = (h.R + kTileM - 1) / kTileM;
+    const int n_slices = umma_slices(h.R, h.V, sm_count);
+    int grid = sm_count;
+    if (nM == 1) {
+        int units = (h.V + 15) / 16;
+        if (grid > units) grid = units;
+    }
+    Partials P = partials_carve(s.partials, (size_t)h.R, (size_t)n_slices);
+
+    HeadArgs hk = h;
+    const void *hid_base = h.hidden;
+    int hid_rows = h.n_src > 0 ? h.n_src : h.R;
+    if (h.row_idx) {
+        // the tensor-map copy cannot follow an index list: pack the gathered rows first
+        const int rows_padded = nM * kTileM;
+        gather_rows_kernel<<<rows_padded, 128, 0, stream>>>(h, (uint4 *)gather_buf, rows_padded, t.stat);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        hid_base = gather_buf;
+        hid_rows = rows_padded;
+        hk.row_idx = nullptr;
+    }
+    CUtensorMap tm_h, tm_w32, tm_w16, tm_w256;
+    if (!make_map(&tm_h, hid_base, hid_rows, h.d, kTileM) || !make_map(&tm_w32, h.W, h.V, h.d, 32) ||
+        !make_map(&tm_w16, h.W, h.V, h.d, 16) || !make_map(&tm_w256, h.W, h.V, h.d, kTileNMax))
+        return cudaErrorInvalidValue;
+    head_umma_kernel<<<grid, kThreads, kDynSmem, stream>>>(tm_h, tm_w32, tm_w16, tm_w256, hk, t, P, s.ticket, nM,
+                                                           n_slices);
+    e = cudaGetLastError();
+    if (e != cudaSuccess || nM == 1) return e;
+    const int fin_grid = (h.R + 7) / 8;
+    head_finalize_kernel<<<fin_grid, 256, 0, stream>>>(hk, t, P, s.ticket, n_slices);
+    return cudaGetLastError();
+}
+
+}  // namespace rstitch
