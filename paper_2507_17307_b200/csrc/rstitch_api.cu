@@ -34,9 +34,17 @@ constexpr int kMaxRows = 16384;
 
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-size_t ws_bytes_for(int R)
+constexpr int kGemvMaxRows = 4;      // above this the CUDA-core kernel stops keeping up with HBM
+
+size_t ws_partials_bytes(int R, int V)
 {
-    return kWsHeader + partials_bytes((size_t)(R > 0 ? R : 1), (size_t)kMaxSlices);
+    return partials_bytes((size_t)(R > 0 ? R : 1), max_slices_for(V));
+}
+
+// [header][partials][gather buffer of the tensor-core kernel]
+size_t ws_bytes_for(int R, int d, int V)
+{
+    return kWsHeader + ws_partials_bytes(R, V) + ((umma_gather_bytes(R > 0 ? R : 1, d) + 255) / 256) * 256;
 }
 
 int shape_status(int R, int d, int V)
@@ -48,7 +56,10 @@ int shape_status(int R, int d, int V)
 
 int grow_handle(rstitch_handle_s *h, int R, int d, int V)
 {
-    size_t need = ws_bytes_for(R);
+    if (R < h->maxR) R = h->maxR;          // the layout depends on all three: never shrink any of them
+    if (d < h->max_d) d = h->max_d;
+    if (V < h->maxV) V = h->maxV;
+    size_t need = ws_bytes_for(R, d, V);
     if (need > h->ws_bytes) {
         if (h->ws) { if (cudaDeviceSynchronize() != cudaSuccess) return RSTITCH_ERR_CUDA; cudaFree(h->ws); h->ws = nullptr; h->ws_bytes = 0; }
         if (cudaMalloc(&h->ws, need) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
@@ -106,7 +117,8 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a)
         !aligned(a->llm_span, 4) || !aligned(a->llm_row_off, 4))
         return RSTITCH_ERR_BAD_ALIGN;
     if (a->workspace) {
-        if (!aligned(a->workspace, 256) || a->workspace_bytes < ws_bytes_for(a->R)) return RSTITCH_ERR_WORKSPACE;
+        if (!aligned(a->workspace, 256) || a->workspace_bytes < ws_bytes_for(a->R, a->d, a->V))
+            return RSTITCH_ERR_WORKSPACE;
     } else if (a->R > h->maxR || a->d > h->max_d || a->V > h->maxV) {
         return RSTITCH_ERR_UNSUPPORTED_SHAPE;
     }
@@ -115,8 +127,10 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a)
 
 bool use_umma(int R, int d, int V, uint32_t flags)
 {
-    (void)R; (void)d; (void)V; (void)flags;
-    return false;
+    if (flags & RSTITCH_PATH_GEMV) return false;
+    if (!umma_shape_ok(R, d, V)) return false;       // tiny shapes stay on the streaming kernel
+    if (flags & RSTITCH_PATH_UMMA) return true;
+    return R > kGemvMaxRows;
 }
 
 }  // namespace
@@ -145,7 +159,7 @@ const char *rstitch_path_name(int R, int d, int V, uint32_t flags)
 size_t rstitch_workspace_bytes(int R, int d, int V)
 {
     if (shape_status(R, d, V) != RSTITCH_OK) return 0;
-    return ws_bytes_for(R);
+    return ws_bytes_for(R, d, V);
 }
 
 int rstitch_create(rstitch_handle_t *out, int maxR, int max_d, int maxV)
@@ -204,12 +218,20 @@ int rstitch_route_ex(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_str
     ta.llm_span = a->llm_span; ta.llm_row_off = a->llm_row_off;
     ta.stat = h->stat;
 
-    Scratch sc = scratch_carve(a->workspace ? a->workspace : h->ws);
+    void *ws = a->workspace ? a->workspace : h->ws;
+    Scratch sc = scratch_carve(ws);
     if (a->workspace) {
         // caller scratch: the ticket must start at zero
         if (cudaMemsetAsync(sc.ticket, 0, sizeof(unsigned), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
     }
-    cudaError_t e = launch_head_gemv(ha, ta, sc, h->sm_count, stream);
+    cudaError_t e;
+    if (use_umma(a->R, a->d, a->V, a->flags)) {
+        // the partials region is sized for the shape the scratch was made for
+        size_t part = a->workspace ? ws_partials_bytes(a->R, a->V) : ws_partials_bytes(h->maxR, h->maxV);
+        e = launch_head_umma(ha, ta, sc, (char *)ws + kWsHeader + part, h->sm_count, stream);
+    } else {
+        e = launch_head_gemv(ha, ta, sc, h->sm_count, stream);
+    }
     if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
     return RSTITCH_OK;
 }

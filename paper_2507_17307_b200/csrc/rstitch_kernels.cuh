@@ -34,6 +34,20 @@ __host__ inline Scratch scratch_carve(void *ws)
 cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch &s, int sm_count,
                              cudaStream_t stream);
 
+// Tensor-core kernel (tcgen05 + tensor memory): any row count; the choice between the two is the
+// caller's.  gather_buf (umma_gather_bytes(R, d) bytes, 256-byte aligned) is used only with row_idx.
+bool        umma_shape_ok(int R, int d, int V);
+size_t      umma_gather_bytes(int R, int d);
+cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
+                             int sm_count, cudaStream_t stream);
+
+// Upper bound on the partials per row of any kernel for a vocabulary of V rows.
+__host__ __device__ inline size_t max_slices_for(int V)
+{
+    size_t tiles = ((size_t)(V > 0 ? V : 1) + 255) / 256;
+    return tiles > (size_t)kMaxSlices ? tiles : (size_t)kMaxSlices;
+}
+
 // Stand-alone ordered compaction (S5).
 cudaError_t launch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, DevStat *stat,
                            int32_t *block_counts /* scratch for B > one block's reach, or null */,

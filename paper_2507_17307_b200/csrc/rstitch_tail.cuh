@@ -64,25 +64,59 @@ struct TailArgs {
     DevStat *stat;
 };
 
-// Merge the n_slices partials of every row in a fixed order (lanes stride over slices, then a
-// butterfly), write ent_out / tok_out.  One warp per row.
+// Writes ent_out / tok_out of one row from its merged statistics.
+__device__ __forceinline__ void tail_emit_row(const Stats &t, int r, const TailArgs &a)
+{
+    float H = logf(t.s) - t.u / t.s;
+    if (H < 0.f) H = 0.f;                      // rounding below zero; NaN stays NaN
+    a.ent_out[r] = H;
+    a.tok_out[r] = (t.bi == INT_MAX || t.bi < 0 || t.bi >= a.V) ? 0 : t.bi;
+    if (H != H) atomicAdd(&a.stat->nan_rows, 1u);
+}
+
+// Merge of slices part, part + parts, ... of one row by one thread, loads issued four at a time.
+__device__ __forceinline__ Stats tail_merge_strided(const Partials &P, size_t row_base, int n_slices,
+                                                    int part, int parts)
+{
+    Stats t = stats_empty();
+    int c = part;
+    for (; c + 3 * parts < n_slices; c += 4 * parts) {
+        Stats p0 = partial_load(P, row_base + c);
+        Stats p1 = partial_load(P, row_base + c + parts);
+        Stats p2 = partial_load(P, row_base + c + 2 * parts);
+        Stats p3 = partial_load(P, row_base + c + 3 * parts);
+        stats_merge(p0, p1);
+        stats_merge(p2, p3);
+        stats_merge(p0, p2);
+        stats_merge(t, p0);
+    }
+    for (; c < n_slices; c += parts) {
+        Stats p = partial_load(P, row_base + c);
+        stats_merge(t, p);
+    }
+    return t;
+}
+
+// Merge the n_slices partials of every row in a fixed order and write ent_out / tok_out.  A row is
+// shared by `parts` adjacent lanes (a power of two, as many as the block can spare for the row
+// count), each taking a strided subset of the slices; a butterfly over the group finishes the row.
 __device__ inline void tail_finalize_rows(const Partials &P, int n_slices, const TailArgs &a)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    for (int r = warp; r < a.R; r += nwarps) {
-        Stats t = stats_empty();
-        for (int c = lane; c < n_slices; c += 32) {
-            Stats p = partial_load(P, (size_t)r * n_slices + c);
+    int parts = 32;
+    while (parts > 1 && a.R * parts > (int)blockDim.x) parts >>= 1;
+    const int rows_per_pass = (int)blockDim.x / parts;
+    const int part = threadIdx.x & (parts - 1);
+    const int sub = threadIdx.x / parts;
+    const bool in_pass = sub < rows_per_pass;          // blockDim.x need not be a multiple of parts
+    for (int r0 = 0; r0 < a.R; r0 += rows_per_pass) {
+        const int r = r0 + sub;
+        const bool act = in_pass && r < a.R;
+        Stats t = act ? tail_merge_strided(P, (size_t)r * n_slices, n_slices, part, parts) : stats_empty();
+        for (int o = parts >> 1; o > 0; o >>= 1) {     // whole warp takes part: same trip count everywhere
+            Stats p = stats_shfl_xor(t, o);
             stats_merge(t, p);
         }
-        stats_warp_allmerge(t);
-        if (lane == 0) {
-            float H = logf(t.s) - t.u / t.s;
-            if (H < 0.f) H = 0.f;                      // rounding below zero; NaN stays NaN
-            a.ent_out[r] = H;
-            a.tok_out[r] = (t.bi == INT_MAX || t.bi < 0 || t.bi >= a.V) ? 0 : t.bi;
-            if (H != H) atomicAdd(&a.stat->nan_rows, 1u);
-        }
+        if (act && part == 0) tail_emit_row(t, r, a);
     }
 }
 

@@ -324,19 +324,9 @@ head_finalize_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (r < R_live) {
-        Stats st = stats_empty();
-        for (int c = lane; c < n_slices; c += 32) {
-            Stats p = partial_load(P, (size_t)r * n_slices + c);
-            stats_merge(st, p);
-        }
+        Stats st = tail_merge_strided(P, (size_t)r * n_slices, n_slices, lane, 32);
         stats_warp_allmerge(st);
-        if (lane == 0) {
-            float H = logf(st.s) - st.u / st.s;
-            if (H < 0.f) H = 0.f;
-            t.ent_out[r] = H;
-            t.tok_out[r] = (st.bi == INT_MAX || st.bi < 0 || st.bi >= t.V) ? 0 : st.bi;
-            if (H != H) atomicAdd(&t.stat->nan_rows, 1u);
-        }
+        if (lane == 0) tail_emit_row(st, r, t);
     }
     __threadfence();
     __syncthreads();
@@ -424,11 +414,6 @@ bool umma_shape_ok(int R, int d, int V)
     return R >= 1 && d >= kTileK && V >= kTileNMax && encode_fn() != nullptr;
 }
 
-int umma_slices(int R, int V, int sm_count)
-{
-    return R <= kTileM ? sm_count : (V + kTileNMax - 1) / kTileNMax;
-}
-
 size_t umma_gather_bytes(int R, int d)
 {
     size_t rows = (size_t)((R + kTileM - 1) / kTileM) * kTileM;
@@ -448,12 +433,13 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
         configured[dev] = true;
     }
     const int nM = (h.R + kTileM - 1) / kTileM;
-    const int n_slices = umma_slices(h.R, h.V, sm_count);
     int grid = sm_count;
+    if (grid > kMaxSlices) grid = kMaxSlices;
     if (nM == 1) {
         int units = (h.V + 15) / 16;
         if (grid > units) grid = units;
     }
+    const int n_slices = nM == 1 ? grid : (h.V + kTileNMax - 1) / kTileNMax;
     Partials P = partials_carve(s.partials, (size_t)h.R, (size_t)n_slices);
 
     HeadArgs hk = h;

@@ -72,6 +72,73 @@ def test_reduced_vocab_workloads(rs, handle, oracle, name, V, B):
         assert 0.0 <= min(rates) and max(rates) <= 1.0
 
 
+# ---- the tensor-core kernel, forced, on shapes that span several tiles and ragged tails ----------
+@pytest.mark.parametrize("B,d,V", [
+    (1, 64, 256), (5, 64, 1000), (16, 128, 4097), (17, 72, 2053), (64, 256, 6007), (128, 192, 3001),
+    (3, 1536, 9001), (33, 512, 40009),
+    (129, 64, 777), (200, 136, 2500), (300, 256, 4099), (544, 320, 1031),
+])
+def test_tensor_core_path_shapes(rs, handle, oracle, B, d, V):
+    assert rs.path_name(B, d, V, rs.PATH_UMMA) == "umma"
+    w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=d, V=V, seed=9000 + B + d + V,
+                   sigma_w=0.5 / math.sqrt(d))
+    check_case(rs, handle, oracle, w, [0, 1], flags=rs.PATH_UMMA)
+
+
+def test_tensor_core_path_gather_live_count_and_spans(rs, handle, oracle):
+    # row gather + device-side live row count, then multi-row spans over several M tiles
+    w = gen.scaled(gen.WORKLOADS["c4_llm_b64"], V=3000, d=512, B=64)
+    w_bits = gen.make_w_head(w)
+    w_dev = to_dev_bf16(w_bits)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    row_idx = np.array([3, 9, 10, 31, 40, 63, 0, 0], dtype=np.int32)
+    live = 6
+    ref = oracle.route(hid, w_bits, w.tau_nats, row_idx=row_idx[:live])
+    gpu = run_gpu(handle, hid, w_dev, w.tau_nats, row_idx=row_idx, n_rows_dev=live, R=8, flags=rs.PATH_UMMA)
+    compare(gpu, ref, w.tau_nats, live, live)
+    assert (gpu["tok"][live:8] == -1).all() and (gpu["ent"][live:8] == -1.0).all()
+    bad = np.array([1, 64, -5, 2], dtype=np.int32)
+    gpu = run_gpu(handle, hid, w_dev, w.tau_nats, row_idx=bad, flags=rs.PATH_UMMA)
+    ref = oracle.route(hid, w_bits, w.tau_nats, row_idx=np.array([1, 0, 0, 2], dtype=np.int32))
+    compare(gpu, ref, w.tau_nats, 4, 4)
+    assert rs.last_status(handle)["bad_row_idx"] == 2
+
+    w = gen.scaled(gen.WORKLOADS["c5_catchup"], V=2500, d=320, B=40)
+    w_bits = gen.make_w_head(w)
+    k = gen.make_spans(w, 0)
+    R = int(k.sum())
+    assert R > 128
+    row_seq = np.repeat(np.arange(w.B, dtype=np.int32), k)
+    hid, _ = gen.make_hidden(w, w_bits, 0, rows=R)
+    seq_len, kv_len = gen.make_kv_state(w, 0, span=k)
+    ref = oracle.route(hid, w_bits, w.tau_nats, row_seq=row_seq, B=w.B, seq_len=seq_len, kv_len=kv_len)
+    gpu = run_gpu(handle, hid, to_dev_bf16(w_bits), w.tau_nats, row_seq=row_seq, B=w.B,
+                  seq_len=seq_len, kv_len=kv_len, flags=rs.PATH_UMMA)
+    compare(gpu, ref, w.tau_nats, R, w.B, row_seq=row_seq, oracle=oracle, seq_len=seq_len, kv_len=kv_len)
+
+
+def test_tensor_core_path_nan_row_and_determinism(rs, handle, oracle):
+    w = gen.scaled(gen.WORKLOADS["c1_tiny"], V=1024, d=64, B=9)
+    w_bits = gen.make_w_head(w)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    hid[4, 5] = 0x7FC0
+    ref = oracle.route(hid, w_bits, 100.0)
+    a = run_gpu(handle, hid, to_dev_bf16(w_bits), 100.0, flags=rs.PATH_UMMA)
+    compare(a, ref, 100.0, 9, 9)
+    assert a["mask"][:9].tolist() == [0, 0, 0, 0, 1, 0, 0, 0, 0] and a["tok"][4] == 0
+    assert rs.last_status(handle)["nan_rows"] == 1
+    b = run_gpu(handle, hid, to_dev_bf16(w_bits), 100.0, flags=rs.PATH_UMMA)
+    for k in a:
+        assert np.array_equal(a[k].view(np.uint8), b[k].view(np.uint8)), k
+
+
+def test_path_choice(rs):
+    assert rs.path_name(1, 1536, 151936) == "gemv" and rs.path_name(4, 3584, 152064) == "gemv"
+    assert rs.path_name(16, 3584, 152064) == "umma" and rs.path_name(544, 5120, 152064) == "umma"
+    assert rs.path_name(64, 32, 4096) == "gemv"          # too small for the tensor-core tiles
+    assert rs.path_name(64, 1536, 151936, rs.PATH_GEMV) == "gemv"
+
+
 def test_all_routed_none_routed_and_threshold_ends(rs, handle, oracle):
     w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], V=2048, d=128, B=64, sigma_w=0.05)
     w_bits = gen.make_w_head(w)
