@@ -120,7 +120,7 @@ typedef struct rstitch_devstat_s {
     uint32_t bad_span;      /* routed sequences with seq_len - kv_len < 1 */
     uint32_t timeouts;      /* bounded device-side waits that gave up */
     uint32_t timeout_site;  /* where the last one gave up (kernel-internal site id) */
-    uint32_t launches;      /* kernels launched through this handle */
+    uint32_t launches;      /* kernels enqueued through this handle (counted on the host) */
     uint32_t reserved[2];
 } rstitch_devstat_t;
 

@@ -25,6 +25,7 @@ struct rstitch_handle_s {
     void    *st_hidden = nullptr;  size_t st_hidden_bytes = 0;
     void    *st_out    = nullptr;  size_t st_out_bytes = 0;
     cudaStream_t last_stream = nullptr;
+    unsigned launch_count = 0;           // kernels enqueued since the status word was last read
 };
 
 namespace {
@@ -225,13 +226,15 @@ int rstitch_route_ex(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_str
         if (cudaMemsetAsync(sc.ticket, 0, sizeof(unsigned), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
     }
     cudaError_t e;
+    int launched = 0;
     if (use_umma(a->R, a->d, a->V, a->flags)) {
         // the partials region is sized for the shape the scratch was made for
         size_t part = a->workspace ? ws_partials_bytes(a->R, a->V) : ws_partials_bytes(h->maxR, h->maxV);
-        e = launch_head_umma(ha, ta, sc, (char *)ws + kWsHeader + part, h->sm_count, stream);
+        e = launch_head_umma(ha, ta, sc, (char *)ws + kWsHeader + part, h->sm_count, stream, &launched);
     } else {
-        e = launch_head_gemv(ha, ta, sc, h->sm_count, stream);
+        e = launch_head_gemv(ha, ta, sc, h->sm_count, stream, &launched);
     }
+    h->launch_count += (unsigned)launched;
     if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
     return RSTITCH_OK;
 }
@@ -330,7 +333,9 @@ int rstitch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, vo
         tiles = h->tile_counts;
     }
     h->last_stream = stream;
-    cudaError_t e = launch_compact(mask, B, idx, count, h->stat, tiles, stream);
+    int launched = 0;
+    cudaError_t e = launch_compact(mask, B, idx, count, h->stat, tiles, stream, &launched);
+    h->launch_count += (unsigned)launched;
     if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
     return RSTITCH_OK;
 }
@@ -349,6 +354,8 @@ int rstitch_last_status(rstitch_handle_t h, rstitch_devstat_t *out)
     if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
     if (cudaMemcpy(out, h->stat, sizeof(DevStat), cudaMemcpyDeviceToHost) != cudaSuccess ||
         cudaMemset(h->stat, 0, sizeof(DevStat)) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    out->launches = h->launch_count;     // counted on the host as the kernels are enqueued
+    h->launch_count = 0;
     return out->timeouts ? RSTITCH_ERR_TIMEOUT : RSTITCH_OK;
 }
 

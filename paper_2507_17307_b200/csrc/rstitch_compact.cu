@@ -97,12 +97,14 @@ compact_scatter_kernel(const uint8_t *mask, int B, const int32_t *tile_offsets, 
 }  // namespace
 
 cudaError_t launch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, DevStat *stat,
-                           int32_t *block_counts, cudaStream_t stream)
+                           int32_t *block_counts, cudaStream_t stream, int *launched)
 {
     if (B <= kCompactOneBlockMax || block_counts == nullptr) {
         compact_one_block_kernel<<<1, kThreads, 0, stream>>>(mask, B, idx, count, stat);
+        *launched = 1;
         return cudaGetLastError();
     }
+    *launched = 3;
     int n_tiles = (B + kCompactTile - 1) / kCompactTile;
     compact_count_kernel<<<n_tiles, kThreads, 0, stream>>>(mask, B, block_counts);
     compact_scan_kernel<<<1, kThreads, 0, stream>>>(block_counts, n_tiles, count);

@@ -216,10 +216,7 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
     tail_finalize_rows(P, n_slices, ta);
     __syncthreads();
     tail_route(ta, s_tail);
-    if (threadIdx.x == 0) {
-        *ticket = 0u;
-        atomicAdd(&t.stat->launches, 1u);
-    }
+    if (threadIdx.x == 0) *ticket = 0u;
 }
 
 struct Plan { int RT, VR, n_slots, hid_bytes; size_t smem; };
@@ -278,8 +275,9 @@ cudaError_t launch_rt(const HeadArgs &h, const TailArgs &t, const Scratch &s, co
 }  // namespace
 
 cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch &s, int sm_count,
-                             cudaStream_t stream)
+                             cudaStream_t stream, int *launched)
 {
+    if (launched) *launched = 1;
     Plan p = make_plan(h.R, h.d);
     if (p.n_slots < 1) return cudaErrorInvalidValue;
     int grid = sm_count;

@@ -31,15 +31,16 @@ __host__ inline Scratch scratch_carve(void *ws)
 }
 
 // CUDA-core streaming kernel: split-V GEMV for a handful of rows.
+// *launched (optional for the streaming kernel) receives the number of kernels enqueued.
 cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch &s, int sm_count,
-                             cudaStream_t stream);
+                             cudaStream_t stream, int *launched = nullptr);
 
 // Tensor-core kernel (tcgen05 + tensor memory): any row count; the choice between the two is the
 // caller's.  gather_buf (umma_gather_bytes(R, d) bytes, 256-byte aligned) is used only with row_idx.
 bool        umma_shape_ok(int R, int d, int V);
 size_t      umma_gather_bytes(int R, int d);
 cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
-                             int sm_count, cudaStream_t stream);
+                             int sm_count, cudaStream_t stream, int *launched);
 
 // Upper bound on the partials per row of any kernel for a vocabulary of V rows.
 __host__ __device__ inline size_t max_slices_for(int V)
@@ -51,7 +52,7 @@ __host__ __device__ inline size_t max_slices_for(int V)
 // Stand-alone ordered compaction (S5).
 cudaError_t launch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, DevStat *stat,
                            int32_t *block_counts /* scratch for B > one block's reach, or null */,
-                           cudaStream_t stream);
+                           cudaStream_t stream, int *launched);
 constexpr int kCompactOneBlockMax = 1 << 16;
 constexpr int kCompactTile        = 4096;     // sequences per block in the multi-block form
 

@@ -29,14 +29,14 @@ namespace rstitch {
 namespace {
 
 constexpr int kThreads   = 192;
-constexpr int kStages    = 4;
+constexpr int kMaxStages = 8;
 constexpr int kTileM     = 128;
 constexpr int kTileNMax  = 256;
 constexpr int kTileK     = 64;                       // bf16 elements = one 128-byte swizzle row
 constexpr int kABytes    = kTileM * kTileK * 2;      // 16 KB
 constexpr int kBBytes    = kTileNMax * kTileK * 2;   // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kDynSmem   = kStages * kStageBytes + 1024;   // + slack to align the ring to 1024 B
+constexpr int kRingBytes = 4 * (kABytes + kBBytes);        // 192 KB, cut into as many stages as fit
+constexpr int kDynSmem   = kRingBytes + 1024;              // + slack to align the ring to 1024 B
 constexpr int kTmemCols  = 512;
 
 struct Item { int v0, N, m; };
@@ -49,7 +49,9 @@ struct Schedule {
     // several M tiles
     int n_items;
 
-    __device__ void init(int V_, int nM_, int grid_, int cta_)
+    // tiles_per_block: the same for every block (from the largest range), so that no block's
+    // tile exceeds the tile size the shared-memory stages were laid out for
+    __device__ void init(int V_, int nM_, int grid_, int cta_, int tiles_per_block)
     {
         V = V_; nM = nM_; grid = grid_; cta = cta_;
         if (nM == 1) {
@@ -57,7 +59,7 @@ struct Schedule {
             u_begin = (int)(units * cta / grid);
             int u_end = (int)(units * (cta + 1) / grid);
             nu = u_end - u_begin;
-            n_tiles = (nu + 15) / 16;
+            n_tiles = tiles_per_block;
             n_items = n_tiles;
         } else {
             int nVT = (V + kTileNMax - 1) / kTileNMax;
@@ -123,13 +125,26 @@ __device__ __forceinline__ void fold_chunk(Stats &st, const float (&z)[32], int 
     st.u += u;
 }
 
+// Tensor maps over W_head with boxes of 16, 32, 64, 128 and 256 rows: a tile of N rows (a multiple
+// of 16) is fetched with one copy per set bit of N / 16, largest first.  Few large copies matter:
+// a copy of a few KB costs the TMA unit about as much time as one of 16 KB.
+struct WMaps { CUtensorMap box[5]; };
+
+// Launch geometry computed on the host.
+struct UmmaPlan {
+    int nM, n_slices;
+    int a_rows;            // hidden rows fetched per k-step (the MMA still reads 128)
+    int n_stages, a_bytes, stage_bytes;
+    int tiles_per_block;   // one M tile only
+};
+
 __global__ void __launch_bounds__(kThreads, 1)
-head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_constant__ CUtensorMap tm_w32,
-                 const __grid_constant__ CUtensorMap tm_w16, const __grid_constant__ CUtensorMap tm_w256,
-                 HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int nM, int n_slices)
+head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_constant__ WMaps tm_w,
+                 HeadArgs h, TailArgs t, Partials P, unsigned *ticket, UmmaPlan plan)
 {
     extern __shared__ unsigned char dyn_smem_raw[];
-    __shared__ __align__(8) uint64_t s_full[kStages], s_empty[kStages];
+    __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
+    const int nM = plan.nM, n_slices = plan.n_slices, n_stages = plan.n_stages;
     __shared__ __align__(8) uint64_t s_acc_full[2], s_acc_empty[2], s_done;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_tail[66];
@@ -142,11 +157,11 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
 
     Schedule sch;
-    sch.init(h.V, nM, gridDim.x, blockIdx.x);
+    sch.init(h.V, nM, gridDim.x, blockIdx.x, plan.tiles_per_block);
 
     if (threadIdx.x == 0) {
         s_abort = 0; s_zero = 0;
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             ptx::mbar_init(ptx::smem_u32(&s_full[s]), 1);
             ptx::mbar_init(ptx::smem_u32(&s_empty[s]), 1);
         }
@@ -157,7 +172,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
         ptx::mbar_init(ptx::smem_u32(&s_done), 1);
         ptx::mbar_fence_init();
         ptx::prefetch_tmap(&tm_hidden);
-        ptx::prefetch_tmap(nM == 1 ? &tm_w32 : &tm_w256);
+        ptx::prefetch_tmap(&tm_w.box[4]);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(&s_tmem_base), kTmemCols);
@@ -182,28 +197,30 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                         break;
                     }
                     const uint32_t full = ptx::smem_u32(&s_full[stage]);
-                    const uint32_t a_dst = ring + (uint32_t)stage * kStageBytes;
-                    const uint32_t b_dst = a_dst + kABytes;
-                    ptx::mbar_arrive_expect_tx(full, (uint32_t)(kABytes + it.N * kTileK * 2));
+                    const uint32_t a_dst = ring + (uint32_t)(stage * plan.stage_bytes);
+                    const uint32_t b_dst = a_dst + (uint32_t)plan.a_bytes;
+                    // only the first a_rows rows of the hidden tile are fetched; the MMA reads all 128,
+                    // and what the stale rows produce lands in accumulator rows nobody looks at
+                    ptx::mbar_arrive_expect_tx(full, (uint32_t)((plan.a_rows + it.N) * kTileK * 2));
                     ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, it.m * kTileM, full);
-                    if (it.N == kTileNMax) {
-                        ptx::tma_g2s_2d(b_dst, &tm_w256, ks * kTileK, it.v0, full);
-                    } else {
-                        int r = 0;
-                        for (; r + 32 <= it.N; r += 32)
-                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w32, ks * kTileK, it.v0 + r, full);
-                        if (r < it.N)
-                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w16, ks * kTileK, it.v0 + r, full);
+                    int r = 0;
+#pragma unroll
+                    for (int b = 4; b >= 0; --b) {
+                        const int rows = 16 << b;
+                        if (it.N - r >= rows) {
+                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK, it.v0 + r, full);
+                            r += rows;
+                        }
                     }
                     ++issued;
-                    if (++stage == kStages) { stage = 0; ++round; }
+                    if (++stage == n_stages) { stage = 0; ++round; }
                 }
             }
             if (s_abort) {
                 // no copy may still be landing in this block's shared memory when it exits
-                int first = issued > kStages ? issued - kStages : 0;
+                int first = issued > n_stages ? issued - n_stages : 0;
                 for (int q = first; q < issued; ++q)
-                    ptx::mbar_wait(ptx::smem_u32(&s_full[q % kStages]), (uint32_t)((q / kStages) & 1), &s_zero);
+                    ptx::mbar_wait(ptx::smem_u32(&s_full[q % n_stages]), (uint32_t)((q / n_stages) & 1), &s_zero);
             }
         }
         __syncwarp();
@@ -229,15 +246,15 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                         break;
                     }
                     ptx::tc_fence_after_sync();
-                    const uint32_t a_src = ring + (uint32_t)stage * kStageBytes;
+                    const uint32_t a_src = ring + (uint32_t)(stage * plan.stage_bytes);
                     const uint64_t a_desc = ptx::smem_desc_sw128(a_src);
-                    const uint64_t b_desc = ptx::smem_desc_sw128(a_src + kABytes);
+                    const uint64_t b_desc = ptx::smem_desc_sw128(a_src + (uint32_t)plan.a_bytes);
 #pragma unroll
                     for (int kk = 0; kk < kTileK / 16; ++kk)     // 32 bytes along K per instruction
                         ptx::umma_bf16(d_tmem, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc,
                                        (uint32_t)((ks | kk) != 0));
                     ptx::umma_commit(ptx::smem_u32(&s_empty[stage]));      // frees the stage when the MMAs are done
-                    if (++stage == kStages) { stage = 0; ++round; }
+                    if (++stage == n_stages) { stage = 0; ++round; }
                 }
                 if (live) ptx::umma_commit(ptx::smem_u32(&s_acc_full[buf]));   // accumulator complete
             }
@@ -306,10 +323,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     tail_finalize_rows(P, n_slices, ta);
     __syncthreads();
     tail_route(ta, s_tail);
-    if (threadIdx.x == 0) {
-        *ticket = 0u;
-        atomicAdd(&t.stat->launches, 1u);
-    }
+    if (threadIdx.x == 0) *ticket = 0u;
 }
 
 // Several M tiles: one warp per row merges that row's per-tile partials; the last block done
@@ -341,10 +355,7 @@ head_finalize_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n
     ta.R = R_live;
     if (h.n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
     tail_route(ta, s_tail);
-    if (threadIdx.x == 0) {
-        *ticket = 0u;
-        atomicAdd(&t.stat->launches, 1u);
-    }
+    if (threadIdx.x == 0) *ticket = 0u;
 }
 
 // hidden[row_idx[r]] -> packed[r] (zero for rows past the live count or with a bad index).
@@ -421,8 +432,9 @@ size_t umma_gather_bytes(int R, int d)
 }
 
 cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
-                             int sm_count, cudaStream_t stream)
+                             int sm_count, cudaStream_t stream, int *launched)
 {
+    *launched = 0;
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -432,40 +444,59 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    const int nM = (h.R + kTileM - 1) / kTileM;
+    UmmaPlan plan;
+    plan.nM = (h.R + kTileM - 1) / kTileM;
     int grid = sm_count;
     if (grid > kMaxSlices) grid = kMaxSlices;
-    if (nM == 1) {
+    int n_max = kTileNMax;
+    plan.tiles_per_block = 0;
+    if (plan.nM == 1) {
         int units = (h.V + 15) / 16;
         if (grid > units) grid = units;
+        int nu = (units + grid - 1) / grid;              // largest range of any block, in 16-row units
+        plan.tiles_per_block = (nu + 15) / 16;
+        n_max = ((nu + plan.tiles_per_block - 1) / plan.tiles_per_block) * 16;
     }
-    const int n_slices = nM == 1 ? grid : (h.V + kTileNMax - 1) / kTileNMax;
-    Partials P = partials_carve(s.partials, (size_t)h.R, (size_t)n_slices);
+    plan.n_slices = plan.nM == 1 ? grid : (h.V + kTileNMax - 1) / kTileNMax;
+    // Stage = the hidden rows actually fetched + the largest W tile of this launch.  The MMA reads
+    // 128 hidden rows from the stage's start whatever was fetched, so the last stage keeps that
+    // much room inside the ring.
+    plan.a_rows = plan.nM == 1 ? ((h.R + 7) / 8) * 8 : kTileM;
+    plan.a_bytes = ((plan.a_rows * kTileK * 2 + 1023) / 1024) * 1024;
+    plan.stage_bytes = plan.a_bytes + n_max * kTileK * 2;
+    plan.n_stages = (kRingBytes - (kABytes - plan.a_bytes)) / plan.stage_bytes;
+    if (plan.n_stages > kMaxStages) plan.n_stages = kMaxStages;
+    Partials P = partials_carve(s.partials, (size_t)h.R, (size_t)plan.n_slices);
 
     HeadArgs hk = h;
     const void *hid_base = h.hidden;
     int hid_rows = h.n_src > 0 ? h.n_src : h.R;
     if (h.row_idx) {
         // the tensor-map copy cannot follow an index list: pack the gathered rows first
-        const int rows_padded = nM * kTileM;
+        const int rows_padded = plan.nM * kTileM;
         gather_rows_kernel<<<rows_padded, 128, 0, stream>>>(h, (uint4 *)gather_buf, rows_padded, t.stat);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
+        ++*launched;
         hid_base = gather_buf;
         hid_rows = rows_padded;
         hk.row_idx = nullptr;
     }
-    CUtensorMap tm_h, tm_w32, tm_w16, tm_w256;
-    if (!make_map(&tm_h, hid_base, hid_rows, h.d, kTileM) || !make_map(&tm_w32, h.W, h.V, h.d, 32) ||
-        !make_map(&tm_w16, h.W, h.V, h.d, 16) || !make_map(&tm_w256, h.W, h.V, h.d, kTileNMax))
-        return cudaErrorInvalidValue;
-    head_umma_kernel<<<grid, kThreads, kDynSmem, stream>>>(tm_h, tm_w32, tm_w16, tm_w256, hk, t, P, s.ticket, nM,
-                                                           n_slices);
+    CUtensorMap tm_h;
+    WMaps tm_w;
+    if (!make_map(&tm_h, hid_base, hid_rows, h.d, plan.a_rows)) return cudaErrorInvalidValue;
+    for (int b = 0; b < 5; ++b)
+        if (!make_map(&tm_w.box[b], h.W, h.V, h.d, 16 << b)) return cudaErrorInvalidValue;
+    head_umma_kernel<<<grid, kThreads, kDynSmem, stream>>>(tm_h, tm_w, hk, t, P, s.ticket, plan);
     e = cudaGetLastError();
-    if (e != cudaSuccess || nM == 1) return e;
+    if (e != cudaSuccess) return e;
+    ++*launched;
+    if (plan.nM == 1) return e;
     const int fin_grid = (h.R + 7) / 8;
-    head_finalize_kernel<<<fin_grid, 256, 0, stream>>>(hk, t, P, s.ticket, n_slices);
-    return cudaGetLastError();
+    head_finalize_kernel<<<fin_grid, 256, 0, stream>>>(hk, t, P, s.ticket, plan.n_slices);
+    e = cudaGetLastError();
+    if (e == cudaSuccess) ++*launched;
+    return e;
 }
 
 }  // namespace rstitch
