@@ -1,0 +1,51 @@
+"""Host-side helpers for running the routing decision on several GPUs.
+
+The path shards by rows: sequences are independent, so every rank decides its own sequences against
+a replicated LM head and there is no data-path collective.  What crosses ranks is only bookkeeping:
+which sequences a rank owns, the slowest rank's time, and the totals.  Nothing here computes any
+part of the decision; it works on CPU tensors with the gloo backend and on CUDA tensors with NCCL.
+"""
+from __future__ import annotations
+
+from typing import Tuple
+
+
+def rank_rows(n_rows: int, rank: int, world: int) -> Tuple[int, int]:
+    """[begin, end) of the sequences rank `rank` decides when n_rows are dealt to `world` ranks
+    in contiguous, balanced blocks (sizes differ by at most one, earlier ranks take the extra)."""
+    if world < 1 or not (0 <= rank < world) or n_rows < 0:
+        raise ValueError("bad sharding arguments")
+    base, extra = divmod(n_rows, world)
+    begin = rank * base + min(rank, extra)
+    return begin, begin + base + (1 if rank < extra else 0)
+
+
+def global_index(local_idx, begin: int):
+    """Sequence ids of a rank's compacted list in the numbering of the whole batch."""
+    return local_idx + begin
+
+
+def reduce_step_stats(ms: float, units: float, launches: int, dist=None, device="cpu"):
+    """(slowest rank's ms, units summed over ranks, launches summed over ranks).
+
+    `dist` is torch.distributed (initialised) or None for a single process."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(ms), float(units), int(launches)
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    s = torch.tensor([units, float(launches)], dtype=torch.float64, device=device)
+    dist.all_reduce(s, op=dist.ReduceOp.SUM)
+    return float(t[0].item()), float(s[0].item()), int(round(float(s[1].item())))
+
+
+def gather_counts(count: int, dist=None, device="cpu"):
+    """Every rank's llm_count, in rank order: the offsets that turn per-rank index lists into one
+    global list are their exclusive prefix sums."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return [int(count)]
+    import torch
+    mine = torch.tensor([int(count)], dtype=torch.int64, device=device)
+    out = [torch.zeros_like(mine) for _ in range(dist.get_world_size())]
+    dist.all_gather(out, mine)
+    return [int(o.item()) for o in out]
