@@ -151,6 +151,18 @@ int rstitch_route_host(rstitch_handle_t h, const void *hidden_host, const void *
                        int32_t *llm_idx_host, int32_t *llm_count_host, void *cuda_stream);
 
 /*
+ * rstitch_route_ex with HOST buffers for everything that changes per step, for a host-driven decode
+ * loop (Algorithm 1 run from the host): in *a, hidden (bf16 [n_src,d]), row_idx, row_seq, seq_len,
+ * kv_len and every output pointer are host pointers (ideally pinned); W_head stays a device pointer.
+ * n_rows_dev and workspace must be NULL (the live row count is simply R, and the scratch is the
+ * handle's).  The inputs are copied to a staging block owned by the handle, the step runs, the
+ * outputs are copied back and the call returns after the stream has been synchronised.  llm_idx
+ * comes back in full (B entries); only the first llm_count are meaningful.  The first call, and any
+ * call needing a larger staging block, allocates device memory.
+ */
+int rstitch_route_ex_host(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_stream);
+
+/*
  * The same decision as rstitch_route (S1-S5, B rows, one decision per row) for callers that cannot
  * allocate device memory.  (The paper has no counterpart; this is a deployment variant.)
  *

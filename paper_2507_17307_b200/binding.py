@@ -20,7 +20,7 @@ PATH_UMMA = 0x20
 EXPORTS = [
     "rstitch_route", "rstitch_route_ex", "rstitch_route_host", "rstitch_create", "rstitch_destroy",
     "rstitch_workspace_bytes", "rstitch_compact", "rstitch_last_status", "rstitch_status_string",
-    "rstitch_path_name", "rstitch_route_static",
+    "rstitch_path_name", "rstitch_route_static", "rstitch_route_ex_host",
 ]
 
 
@@ -72,6 +72,8 @@ def lib():
         L.rstitch_route.restype = i
         L.rstitch_route_ex.argtypes = [vp, C.POINTER(_Args), vp]
         L.rstitch_route_ex.restype = i
+        L.rstitch_route_ex_host.argtypes = [vp, C.POINTER(_Args), vp]
+        L.rstitch_route_ex_host.restype = i
         L.rstitch_route_host.argtypes = [vp, vp, vp, i, i, i, f, vp, vp, vp, vp, vp, vp]
         L.rstitch_route_host.restype = i
         L.rstitch_create.argtypes = [C.POINTER(vp), i, i, i]
@@ -279,6 +281,53 @@ def route_host(handle: Handle, hidden_host, W_head_dev, tau: float, host_out: di
                                   _stream_ptr(stream))
     if st != 0:
         raise RstitchError(st, "rstitch_route_host")
+    return host_out
+
+
+class PreparedHostCall:
+    """rstitch_route_ex_host with its rstitch_args_t filled once: hidden, the optional index arrays
+    and every output are CPU tensors (ideally pinned), W_head a device tensor.  host_out holds 'tok'
+    int32 [R], 'ent' float32 [R], 'mask' uint8 [B], 'llm_idx' int32 [B], 'llm_count' int32 [1] and,
+    with seq_len / kv_len, 'llm_span' int32 [B] and 'llm_row_off' int32 [B + 1]."""
+
+    def __init__(self, handle: Handle, hidden_host, W_head_dev, tau: float, host_out: dict, *, R=None, B=None,
+                 row_idx=None, row_seq=None, seq_len=None, kv_len=None, flags=0, stream=None):
+        n_src, d = int(hidden_host.shape[0]), int(hidden_host.shape[1])
+        if R is None:
+            R = int(row_idx.shape[0]) if row_idx is not None else n_src
+        if B is None:
+            B = R
+        a = _Args()
+        a.hidden, a.W_head = _ptr(hidden_host), _ptr(W_head_dev)
+        a.R, a.B, a.d, a.V, a.n_src = R, B, d, int(W_head_dev.shape[0]), n_src
+        a.tau, a.flags = float(tau), int(flags)
+        a.row_idx, a.row_seq = _ptr(row_idx), _ptr(row_seq)
+        a.seq_len, a.kv_len = _ptr(seq_len), _ptr(kv_len)
+        a.tok_out, a.ent_out, a.route_mask = _ptr(host_out["tok"]), _ptr(host_out["ent"]), _ptr(host_out["mask"])
+        a.llm_idx, a.llm_count = _ptr(host_out["llm_idx"]), _ptr(host_out["llm_count"])
+        a.llm_span, a.llm_row_off = _ptr(host_out.get("llm_span")), _ptr(host_out.get("llm_row_off"))
+        self._keep = (handle, hidden_host, W_head_dev, host_out, row_idx, row_seq, seq_len, kv_len)
+        self.args = a
+        self._ref = C.byref(a)
+        self._h = handle.ptr
+        self._stream = _stream_ptr(stream)
+        self._fn = lib().rstitch_route_ex_host
+        self.out = host_out
+
+    def set_rows(self, R: int, B: Optional[int] = None):
+        """Change the row count between steps (e.g. to the llm_count an earlier call returned)."""
+        self.args.R = int(R)
+        self.args.B = int(R if B is None else B)
+
+    def launch(self) -> int:
+        return self._fn(self._h, self._ref, self._stream)
+
+
+def route_ex_host(handle: Handle, hidden_host, W_head_dev, tau: float, host_out: dict, **kw):
+    """rstitch_route_ex_host, one call; see PreparedHostCall for the arguments."""
+    st = PreparedHostCall(handle, hidden_host, W_head_dev, tau, host_out, **kw).launch()
+    if st != 0:
+        raise RstitchError(st, "rstitch_route_ex_host")
     return host_out
 
 

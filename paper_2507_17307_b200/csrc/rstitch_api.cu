@@ -22,8 +22,7 @@ struct rstitch_handle_s {
     int32_t *tile_counts = nullptr;      // scratch of the multi-block compaction
     int      tile_cap    = 0;
     // staging of rstitch_route_host
-    void    *st_hidden = nullptr;  size_t st_hidden_bytes = 0;
-    void    *st_out    = nullptr;  size_t st_out_bytes = 0;
+    void    *st = nullptr;  size_t st_bytes = 0;     // staging block of the host-buffer calls
     cudaStream_t last_stream = nullptr;
     unsigned launch_count = 0;           // kernels enqueued since the status word was last read
 };
@@ -184,7 +183,7 @@ int rstitch_create(rstitch_handle_t *out, int maxR, int max_d, int maxV)
 int rstitch_destroy(rstitch_handle_t h)
 {
     if (!h) return RSTITCH_OK;
-    cudaFree(h->ws); cudaFree(h->stat); cudaFree(h->tile_counts); cudaFree(h->st_hidden); cudaFree(h->st_out);
+    cudaFree(h->ws); cudaFree(h->stat); cudaFree(h->tile_counts); cudaFree(h->st);
     cudaGetLastError();
     delete h;
     return RSTITCH_OK;
@@ -256,57 +255,96 @@ int rstitch_route(const void *hidden, const void *W_head, int B, int d, int V, f
     return rstitch_route_ex(h, &a, nullptr);
 }
 
+int rstitch_route_ex_host(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_stream)
+{
+    if (!h || !a) return RSTITCH_ERR_INVALID_ARG;
+    if (a->n_rows_dev || a->workspace) return RSTITCH_ERR_INVALID_ARG;     // host-driven: no device-side inputs
+    int st = shape_status(a->R, a->d, a->V);
+    if (st != RSTITCH_OK) return st;
+    if (a->B < 0 || a->n_src < 0 || !a->llm_count) return RSTITCH_ERR_INVALID_ARG;
+    if (a->R > 0 && (!a->hidden || !a->W_head || !a->tok_out || !a->ent_out)) return RSTITCH_ERR_INVALID_ARG;
+    if (a->B > 0 && (!a->route_mask || !a->llm_idx)) return RSTITCH_ERR_INVALID_ARG;
+    if ((a->seq_len == nullptr) != (a->kv_len == nullptr)) return RSTITCH_ERR_INVALID_ARG;
+    if (a->seq_len && a->B > 0 && (!a->llm_span || !a->llm_row_off)) return RSTITCH_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const size_t R = (size_t)a->R, B = (size_t)a->B;
+    const size_t n_src = a->n_src > 0 ? (size_t)a->n_src : R;
+    if (R == 0 || B == 0) {
+        *a->llm_count = 0;
+        if (a->seq_len && a->llm_row_off) a->llm_row_off[0] = 0;
+        if (R == 0) return RSTITCH_OK;
+    }
+
+    // one staging block: inputs first, then the outputs; every piece 256-byte aligned
+    auto up = [](size_t n) { return (n + 255) / 256 * 256; };
+    size_t off = 0;
+    const size_t o_hid = off;  off += up(n_src * a->d * 2);
+    const size_t o_ridx = off; off += up(R * 4);
+    const size_t o_rseq = off; off += up(R * 4);
+    const size_t o_slen = off; off += up(B * 4);
+    const size_t o_klen = off; off += up(B * 4);
+    const size_t o_tok = off;  off += up(R * 4);
+    const size_t o_ent = off;  off += up(R * 4);
+    const size_t o_idx = off;  off += up(B * 4);
+    const size_t o_span = off; off += up(B * 4);
+    const size_t o_roff = off; off += up((B + 1) * 4);
+    const size_t o_cnt = off;  off += 256;
+    const size_t o_msk = off;  off += up(B);
+    if (off > h->st_bytes) {
+        if (h->st) { cudaDeviceSynchronize(); cudaFree(h->st); h->st = nullptr; h->st_bytes = 0; }
+        if (cudaMalloc(&h->st, off) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+        h->st_bytes = off;
+    }
+    char *base = (char *)h->st;
+    auto h2d = [&](size_t o, const void *src, size_t n) {
+        return n == 0 || cudaMemcpyAsync(base + o, src, n, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    };
+    auto d2h = [&](void *dst, size_t o, size_t n) {
+        return n == 0 || cudaMemcpyAsync(dst, base + o, n, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    };
+    bool ok = h2d(o_hid, a->hidden, n_src * a->d * 2);
+    if (ok && a->row_idx) ok = h2d(o_ridx, a->row_idx, R * 4);
+    if (ok && a->row_seq) ok = h2d(o_rseq, a->row_seq, R * 4);
+    if (ok && a->seq_len) ok = h2d(o_slen, a->seq_len, B * 4) && h2d(o_klen, a->kv_len, B * 4);
+    if (!ok) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+
+    rstitch_args_t dv = *a;
+    dv.hidden = base + o_hid;
+    dv.n_src = (int32_t)n_src;
+    dv.row_idx = a->row_idx ? (const int32_t *)(base + o_ridx) : nullptr;
+    dv.row_seq = a->row_seq ? (const int32_t *)(base + o_rseq) : nullptr;
+    dv.seq_len = a->seq_len ? (const int32_t *)(base + o_slen) : nullptr;
+    dv.kv_len  = a->seq_len ? (const int32_t *)(base + o_klen) : nullptr;
+    dv.tok_out = (int32_t *)(base + o_tok);
+    dv.ent_out = (float *)(base + o_ent);
+    dv.llm_idx = (int32_t *)(base + o_idx);
+    dv.llm_span = a->seq_len ? (int32_t *)(base + o_span) : nullptr;
+    dv.llm_row_off = a->seq_len ? (int32_t *)(base + o_roff) : nullptr;
+    dv.llm_count = (int32_t *)(base + o_cnt);
+    dv.route_mask = (uint8_t *)(base + o_msk);
+    st = rstitch_route_ex(h, &dv, cuda_stream);
+    if (st != RSTITCH_OK) return st;
+
+    ok = d2h(a->tok_out, o_tok, R * 4) && d2h(a->ent_out, o_ent, R * 4) && d2h(a->llm_idx, o_idx, B * 4) &&
+         d2h(a->llm_count, o_cnt, 4) && d2h(a->route_mask, o_msk, B);
+    if (ok && a->seq_len) ok = d2h(a->llm_span, o_span, B * 4) && d2h(a->llm_row_off, o_roff, (B + 1) * 4);
+    ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    return RSTITCH_OK;
+}
+
 int rstitch_route_host(rstitch_handle_t h, const void *hidden_host, const void *W_head_dev,
                        int B, int d, int V, float tau, int32_t *tok_host, float *ent_host,
                        uint8_t *mask_host, int32_t *llm_idx_host, int32_t *llm_count_host,
                        void *cuda_stream)
 {
-    if (!h) return RSTITCH_ERR_INVALID_ARG;
-    int st = shape_status(B, d, V);
-    if (st != RSTITCH_OK) return st;
-    if (!llm_count_host) return RSTITCH_ERR_INVALID_ARG;
-    if (B > 0 && (!hidden_host || !W_head_dev || !tok_host || !ent_host || !mask_host || !llm_idx_host))
-        return RSTITCH_ERR_INVALID_ARG;
-    cudaStream_t stream = (cudaStream_t)cuda_stream;
-    if (B == 0) { *llm_count_host = 0; return RSTITCH_OK; }
-
-    // staging: hidden [B,d] bf16 | outputs packed as tok, ent, llm_idx (4 B each), count, mask
-    size_t hid_bytes = (size_t)B * d * 2;
-    size_t out_bytes = (size_t)B * 12 + 16 + (size_t)B;
-    if (hid_bytes > h->st_hidden_bytes) {
-        if (h->st_hidden) { cudaDeviceSynchronize(); cudaFree(h->st_hidden); h->st_hidden = nullptr; h->st_hidden_bytes = 0; }
-        if (cudaMalloc(&h->st_hidden, hid_bytes) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
-        h->st_hidden_bytes = hid_bytes;
-    }
-    if (out_bytes > h->st_out_bytes) {
-        if (h->st_out) { cudaDeviceSynchronize(); cudaFree(h->st_out); h->st_out = nullptr; h->st_out_bytes = 0; }
-        if (cudaMalloc(&h->st_out, out_bytes) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
-        h->st_out_bytes = out_bytes;
-    }
-    char *o = (char *)h->st_out;
-    int32_t *d_tok = (int32_t *)o;
-    float   *d_ent = (float *)(o + (size_t)B * 4);
-    int32_t *d_idx = (int32_t *)(o + (size_t)B * 8);
-    int32_t *d_cnt = (int32_t *)(o + (size_t)B * 12);
-    uint8_t *d_msk = (uint8_t *)(o + (size_t)B * 12 + 16);
-
-    if (cudaMemcpyAsync(h->st_hidden, hidden_host, hid_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
-        { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    if (B < 0) return RSTITCH_ERR_INVALID_ARG;
     rstitch_args_t a;
     std::memset(&a, 0, sizeof a);
-    a.hidden = h->st_hidden; a.W_head = W_head_dev; a.R = B; a.B = B; a.d = d; a.V = V; a.n_src = B; a.tau = tau;
-    a.tok_out = d_tok; a.ent_out = d_ent; a.route_mask = d_msk; a.llm_idx = d_idx; a.llm_count = d_cnt;
-    st = rstitch_route_ex(h, &a, cuda_stream);
-    if (st != RSTITCH_OK) return st;
-    // outputs are contiguous in the staging block: tok | ent | idx | count come back in one copy
-    bool ok = cudaMemcpyAsync(tok_host, d_tok, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
-              cudaMemcpyAsync(ent_host, d_ent, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
-              cudaMemcpyAsync(llm_idx_host, d_idx, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
-              cudaMemcpyAsync(llm_count_host, d_cnt, 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
-              cudaMemcpyAsync(mask_host, d_msk, (size_t)B, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
-              cudaStreamSynchronize(stream) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
-    return RSTITCH_OK;
+    a.hidden = hidden_host; a.W_head = W_head_dev; a.R = B; a.B = B; a.d = d; a.V = V; a.n_src = B; a.tau = tau;
+    a.tok_out = tok_host; a.ent_out = ent_host; a.route_mask = mask_host; a.llm_idx = llm_idx_host;
+    a.llm_count = llm_count_host;
+    return rstitch_route_ex_host(h, &a, cuda_stream);
 }
 
 int rstitch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, void *cuda_stream)

@@ -277,6 +277,45 @@ def test_host_buffer_entry_point(rs, handle, oracle):
     compare(gpu, ref, w.tau_nats, 64, 64)
 
 
+def test_host_buffer_extended_entry_point(rs, handle, oracle):
+    # multi-row spans with everything per-step in host memory, then a row gather driven from the host
+    import torch
+    w = gen.scaled(gen.WORKLOADS["c5_catchup"], V=2500, d=320, B=12)
+    w_bits = gen.make_w_head(w)
+    w_dev = to_dev_bf16(w_bits)
+    k = gen.make_spans(w, 1)
+    R = int(k.sum())
+    row_seq = np.repeat(np.arange(w.B, dtype=np.int32), k)
+    hid, _ = gen.make_hidden(w, w_bits, 1, rows=R)
+    seq_len, kv_len = gen.make_kv_state(w, 1, span=k)
+
+    def host_out(R, B):
+        return {"tok": torch.full((R,), -1, dtype=torch.int32).pin_memory(),
+                "ent": torch.zeros(R, dtype=torch.float32).pin_memory(),
+                "mask": torch.zeros(B, dtype=torch.uint8).pin_memory(),
+                "llm_idx": torch.full((B,), -1, dtype=torch.int32).pin_memory(),
+                "llm_count": torch.zeros(1, dtype=torch.int32).pin_memory(),
+                "llm_span": torch.full((B,), -1, dtype=torch.int32).pin_memory(),
+                "llm_row_off": torch.full((B + 1,), -1, dtype=torch.int32).pin_memory()}
+
+    hh = torch.from_numpy(hid.view(np.int16)).view(torch.bfloat16).pin_memory()
+    out = rs.route_ex_host(handle, hh, w_dev, w.tau_nats, host_out(R, w.B), R=R, B=w.B,
+                           row_seq=torch.from_numpy(row_seq), seq_len=torch.from_numpy(seq_len),
+                           kv_len=torch.from_numpy(kv_len))
+    ref = oracle.route(hid, w_bits, w.tau_nats, row_seq=row_seq, B=w.B, seq_len=seq_len, kv_len=kv_len)
+    gpu = {k_: v.numpy() for k_, v in out.items()}
+    cnt = int(gpu["llm_count"][0])
+    gpu["llm_idx"][cnt:] = -1
+    compare(gpu, ref, w.tau_nats, R, w.B, row_seq=row_seq, oracle=oracle, seq_len=seq_len, kv_len=kv_len)
+
+    row_idx = np.array([5, 0, R - 1, 7, 7], dtype=np.int32)
+    out = rs.route_ex_host(handle, hh, w_dev, w.tau_nats, host_out(5, 5), row_idx=torch.from_numpy(row_idx))
+    ref = oracle.route(hid, w_bits, w.tau_nats, row_idx=row_idx)
+    gpu = {k_: v.numpy() for k_, v in out.items()}
+    gpu["llm_idx"][int(gpu["llm_count"][0]):] = -1
+    compare(gpu, ref, w.tau_nats, 5, 5)
+
+
 def test_caller_workspace(rs, handle, oracle):
     import torch
     w = gen.scaled(gen.WORKLOADS["c3_llm_b4"], V=3001, d=128)
