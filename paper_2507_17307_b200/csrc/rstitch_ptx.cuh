@@ -74,6 +74,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Orders this thread's earlier ordinary (generic-proxy) memory traffic, and what it has observed of
+// other threads', before the asynchronous-proxy operations (bulk copies) it issues next.
+__device__ __forceinline__ void fence_proxy_async_all()
+{
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
+
 // ---- bulk copies ------------------------------------------------------------------------
 // Untiled copy global -> shared; both addresses 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)

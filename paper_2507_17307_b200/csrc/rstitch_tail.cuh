@@ -3,6 +3,7 @@
 // stand-alone compaction kernel.  No block ever waits on another, so nothing here can hang.
 #pragma once
 #include "rstitch_stats.cuh"
+#include "rstitch_ptx.cuh"
 #include <stdint.h>
 
 namespace rstitch {
@@ -118,6 +119,92 @@ __device__ inline void tail_finalize_rows(const Partials &P, int n_slices, const
         }
         if (act && part == 0) tail_emit_row(t, r, a);
     }
+}
+
+// The same finalisation for many rows (tensor-core kernel, up to 128 rows x ~150 slices), where
+// fetching the partials straight from L2 is a chain of dependent round trips.  The partials of a
+// group of rows are first brought into shared memory with five bulk copies (one per statistics
+// array; the rows of a group are contiguous in each), then merged from there without a dependent
+// chain: pass 1 takes the row maximum M and the greedy token, pass 2 sums e^{m_i - M} s_i and
+// e^{m_i - M} (u_i + (m_i - M) s_i), one exponential per partial.
+//   stage / stage_bytes: free shared memory (16-byte aligned); bar: an initialised mbarrier
+//   (count 1) whose completed phases so far number bar_phase.
+// Returns false if a bounded wait ran out (the caller records it).
+__device__ inline bool tail_finalize_rows_staged(const Partials &P, int n_slices, const TailArgs &a,
+                                                 unsigned char *stage, uint32_t stage_bytes, uint64_t *bar,
+                                                 uint32_t bar_phase, volatile int *abort_flag)
+{
+    int parts = 32;
+    while (parts > 1 && a.R * parts > (int)blockDim.x) parts >>= 1;
+    const int part = threadIdx.x & (parts - 1);
+    const int sub = threadIdx.x / parts;
+    const uint32_t row_bytes = (uint32_t)n_slices * 4u;
+    int group = stage_bytes > 80u ? (int)((stage_bytes - 80u) / 5u / row_bytes) & ~3 : 0;   // rows per group
+    if (group > (int)blockDim.x / parts) group = ((int)blockDim.x / parts) & ~3;
+    if (group < 4) {                                                     // no room to stage: read from L2
+        tail_finalize_rows(P, n_slices, a);
+        return true;
+    }
+    const uint32_t region = (((uint32_t)group * row_bytes + 15u) & ~15u);
+    const float *sm_m = (const float *)(stage);
+    const float *sm_s = (const float *)(stage + region);
+    const float *sm_u = (const float *)(stage + 2 * region);
+    const float *sm_bv = (const float *)(stage + 3 * region);
+    const int   *sm_bi = (const int *)(stage + 4 * region);
+    const uint32_t bar_u32 = ptx::smem_u32(bar);
+    bool ok = true;
+    for (int g0 = 0; g0 < a.R; g0 += group, ++bar_phase) {
+        const int rows = (a.R - g0) < group ? (a.R - g0) : group;
+        if (threadIdx.x == 0) {
+            const uint32_t bytes = (((uint32_t)rows * row_bytes + 15u) & ~15u);
+            const size_t off = (size_t)g0 * n_slices;
+            ptx::fence_proxy_async_all();       // the partials were written with ordinary stores
+            ptx::mbar_arrive_expect_tx(bar_u32, 5u * bytes);
+            ptx::bulk_g2s(ptx::smem_u32(sm_m), P.m + off, bytes, bar_u32);
+            ptx::bulk_g2s(ptx::smem_u32(sm_s), P.s + off, bytes, bar_u32);
+            ptx::bulk_g2s(ptx::smem_u32(sm_u), P.u + off, bytes, bar_u32);
+            ptx::bulk_g2s(ptx::smem_u32(sm_bv), P.bv + off, bytes, bar_u32);
+            ptx::bulk_g2s(ptx::smem_u32(sm_bi), P.bi + off, bytes, bar_u32);
+        }
+        if (!ptx::mbar_wait(bar_u32, bar_phase & 1u, abort_flag)) ok = false;
+        const int r = g0 + sub;
+        const bool act = ok && sub < rows;
+        const int base = sub * n_slices;
+        float M = -CUDART_INF_F, bv = -CUDART_INF_F;
+        int bi = INT_MAX;
+        if (act)
+            for (int c = part; c < n_slices; c += parts) {
+                M = fmaxf(M, sm_m[base + c]);
+                argmax_take(bv, bi, sm_bv[base + c], sm_bi[base + c]);
+            }
+        for (int o = parts >> 1; o > 0; o >>= 1) {
+            M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+            float obv = __shfl_xor_sync(0xffffffffu, bv, o);
+            int obi = __shfl_xor_sync(0xffffffffu, bi, o);
+            argmax_take(bv, bi, obv, obi);
+        }
+        float ss = 0.f, uu = 0.f;
+        if (act)
+            for (int c = part; c < n_slices; c += parts) {
+                const float mi = sm_m[base + c];
+                if (mi != -CUDART_INF_F) {
+                    const float dm = mi - M, e = __expf(dm), si = sm_s[base + c];
+                    ss = fmaf(e, si, ss);
+                    uu = fmaf(e, fmaf(dm, si, sm_u[base + c]), uu);
+                }
+            }
+        for (int o = parts >> 1; o > 0; o >>= 1) {
+            ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            uu += __shfl_xor_sync(0xffffffffu, uu, o);
+        }
+        if (act && part == 0) {
+            Stats t;
+            t.m = M; t.s = ss; t.u = uu; t.bv = bv; t.bi = bi;
+            tail_emit_row(t, r, a);
+        }
+        __syncthreads();                        // the stage is reused by the next group
+    }
+    return ok;
 }
 
 // Eq. 2 / Algorithm 1: mask = H > tau (strict); a NaN entropy routes to the LLM.

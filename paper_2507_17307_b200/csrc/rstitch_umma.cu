@@ -93,9 +93,48 @@ __device__ __forceinline__ void raise_abort(volatile int *flag, DevStat *stat, u
     atomicExch(&stat->timeout_site, site);
 }
 
-// Fold up to 32 logits (columns c0 .. c0+31 of the tile, vocabulary index v0 + column) into the
-// row's statistics.  n_valid = how many of them are real vocabulary entries.
-__device__ __forceinline__ void fold_chunk(Stats &st, const float (&z)[32], int n_valid, int vbase)
+// Fold 32 logits (columns c0 .. c0+31 of the tile, vocabulary index vbase + column) into the row's
+// statistics: one rescale of the running sums per chunk, then one ex2 per logit.  Four independent
+// partial maxima / sums keep the dependent chains short: an epilogue warp has a scheduler to itself,
+// so instruction-level parallelism is all the latency hiding there is.
+__device__ __forceinline__ void fold_chunk_full(Stats &st, const float (&z)[32], int vbase)
+{
+    float c0 = fmaxf(z[0], z[4]), c1 = fmaxf(z[1], z[5]), c2 = fmaxf(z[2], z[6]), c3 = fmaxf(z[3], z[7]);
+#pragma unroll
+    for (int i = 8; i < 32; i += 4) {
+        c0 = fmaxf(c0, z[i]); c1 = fmaxf(c1, z[i + 1]); c2 = fmaxf(c2, z[i + 2]); c3 = fmaxf(c3, z[i + 3]);
+    }
+    const float cmax = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));          // fmaxf skips NaN operands
+    const float m_new = fmaxf(st.m, cmax);
+    if (st.m == -CUDART_INF_F) { st.s = 0.f; st.u = 0.f; }
+    else {
+        float dm = st.m - m_new;
+        float a = __expf(dm);
+        st.u = a * (st.u + dm * st.s);
+        st.s = a * st.s;
+    }
+    st.m = m_new;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, u0 = 0.f, u1 = 0.f, u2 = 0.f, u3 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        float d0 = z[i] - m_new, d1 = z[i + 1] - m_new, d2 = z[i + 2] - m_new, d3 = z[i + 3] - m_new;
+        float e0 = __expf(d0), e1 = __expf(d1), e2 = __expf(d2), e3 = __expf(d3);   // NaN logit -> NaN sums
+        s0 += e0; s1 += e1; s2 += e2; s3 += e3;
+        u0 = fmaf(e0, d0, u0); u1 = fmaf(e1, d1, u1); u2 = fmaf(e2, d2, u2); u3 = fmaf(e3, d3, u3);
+    }
+    st.s += (s0 + s1) + (s2 + s3);
+    st.u += (u0 + u1) + (u2 + u3);
+    if (cmax > st.bv) {                       // strictly larger: an earlier chunk keeps a tie
+        int idx = 31;
+#pragma unroll
+        for (int i = 30; i >= 0; --i) idx = (z[i] == cmax) ? i : idx;     // lowest column holding the maximum
+        st.bv = cmax;
+        st.bi = vbase + idx;
+    }
+}
+
+// The same for a chunk with fewer than 32 real vocabulary entries (tile tails).
+__device__ __forceinline__ void fold_chunk_tail(Stats &st, const float (&z)[32], int n_valid, int vbase)
 {
     float cmax = -CUDART_INF_F;
 #pragma unroll
@@ -125,6 +164,12 @@ __device__ __forceinline__ void fold_chunk(Stats &st, const float (&z)[32], int 
     st.u += u;
 }
 
+__device__ __forceinline__ void fold_chunk(Stats &st, const float (&z)[32], int n_valid, int vbase)
+{
+    if (n_valid >= 32) fold_chunk_full(st, z, vbase);     // n_valid is the same in every lane
+    else               fold_chunk_tail(st, z, n_valid, vbase);
+}
+
 // Tensor maps over W_head with boxes of 16, 32, 64, 128 and 256 rows: a tile of N rows (a multiple
 // of 16) is fetched with one copy per set bit of N / 16, largest first.  Few large copies matter:
 // a copy of a few KB costs the TMA unit about as much time as one of 16 KB.
@@ -145,7 +190,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     extern __shared__ unsigned char dyn_smem_raw[];
     __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
     const int nM = plan.nM, n_slices = plan.n_slices, n_stages = plan.n_stages;
-    __shared__ __align__(8) uint64_t s_acc_full[2], s_acc_empty[2], s_done;
+    __shared__ __align__(8) uint64_t s_acc_full[2], s_acc_empty[2], s_done, s_tailbar;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_tail[66];
     __shared__ int s_last, s_abort, s_zero;
@@ -170,6 +215,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
             ptx::mbar_init(ptx::smem_u32(&s_acc_empty[b]), 4);     // one arrival per epilogue warp
         }
         ptx::mbar_init(ptx::smem_u32(&s_done), 1);
+        ptx::mbar_init(ptx::smem_u32(&s_tailbar), 1);
         ptx::mbar_fence_init();
         ptx::prefetch_tmap(&tm_hidden);
         ptx::prefetch_tmap(&tm_w.box[4]);
@@ -320,10 +366,216 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     TailArgs ta = t;
     ta.R = R_live;
     if (h.n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
-    tail_finalize_rows(P, n_slices, ta);
+    // the ring is idle now: stage the partials through it (fast path), or read them from L2
+    if (ta.R > 8) {
+        unsigned char *stage = dyn_smem_raw + (ring - ptx::smem_u32(dyn_smem_raw));
+        if (!tail_finalize_rows_staged(P, n_slices, ta, stage, (uint32_t)kRingBytes, &s_tailbar, 0u, &s_abort) &&
+            threadIdx.x == 0)
+            raise_abort(&s_abort, t.stat, 0x205u);
+    } else {
+        tail_finalize_rows(P, n_slices, ta);
+    }
     __syncthreads();
     tail_route(ta, s_tail);
     if (threadIdx.x == 0) *ticket = 0u;
+}
+
+// ---- several M tiles, two per W tile ------------------------------------------------------------
+// With more than 128 rows the kernel above is fed from L2 and starves: a 128 x 256 accumulator tile
+// needs 48 KB of operands per 512 tensor-pipe cycles.  Here one block works on TWO M tiles against
+// the same W tile, so each 32 KB W stage is used twice (64 KB per 1024 cycles) and the ring looks
+// 50 % further ahead in time.  The 512 tensor-memory columns hold the two accumulators, so there is
+// no second buffer: eight epilogue warps (four per accumulator) drain them while the tensor pipe
+// waits, a few percent of an item.  Work items are (vocabulary tile, pair of M tiles), dealt
+// round-robin with the pairs of one vocabulary tile adjacent (W_head from HBM once, then from L2).
+constexpr int kThreads2    = 320;                          // producer, MMA, 8 epilogue warps
+constexpr int kStages2     = 3;
+constexpr int kStage2Bytes = 2 * kABytes + kBBytes;        // 64 KB
+constexpr int kDynSmem2    = kStages2 * kStage2Bytes + 1024;
+
+struct Item2 { int v0, N, m0, two; };
+
+__device__ __forceinline__ Item2 item2(int q, int nMG, int nM, int V)
+{
+    Item2 it;
+    int vt = q / nMG;
+    int mg = q - vt * nMG;
+    it.m0 = 2 * mg;
+    it.two = (it.m0 + 1 < nM) ? 1 : 0;
+    it.v0 = vt * kTileNMax;
+    int left = V - it.v0;
+    it.N = left >= kTileNMax ? kTileNMax : ((left + 15) / 16) * 16;
+    return it;
+}
+
+__global__ void __launch_bounds__(kThreads2, 1)
+head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_constant__ WMaps tm_w,
+                  HeadArgs h, TailArgs t, Partials P, int nM, int n_slices)
+{
+    extern __shared__ unsigned char dyn_smem_raw[];
+    __shared__ __align__(8) uint64_t s_full[kStages2], s_empty[kStages2];
+    __shared__ __align__(8) uint64_t s_acc_full, s_acc_empty, s_done;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort, s_zero;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ring = (ptx::smem_u32(dyn_smem_raw) + 1023u) & ~1023u;
+    const int nK = (h.d + kTileK - 1) / kTileK;
+    int R_live = h.R;
+    if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
+    const int nMG = (nM + 1) / 2;
+    const int total = ((h.V + kTileNMax - 1) / kTileNMax) * nMG;
+    const int cta = blockIdx.x, grid = gridDim.x;
+    const int n_items = cta < total ? (total - cta + grid - 1) / grid : 0;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0; s_zero = 0;
+        for (int s = 0; s < kStages2; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&s_full[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&s_empty[s]), 1);
+        }
+        ptx::mbar_init(ptx::smem_u32(&s_acc_full), 1);
+        ptx::mbar_init(ptx::smem_u32(&s_acc_empty), 8);        // one arrival per epilogue warp
+        ptx::mbar_init(ptx::smem_u32(&s_done), 1);
+        ptx::mbar_fence_init();
+        ptx::prefetch_tmap(&tm_hidden);
+        ptx::prefetch_tmap(&tm_w.box[4]);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(&s_tmem_base), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = s_tmem_base;
+
+    if (warp == 0) {
+        // ---- producer --------------------------------------------------------------------
+        if (lane == 0) {
+            int stage = 0, round = 0, issued = 0;
+            bool live = true;
+            for (int j = 0; live && j < n_items; ++j) {
+                const Item2 it = item2(cta + j * grid, nMG, nM, h.V);
+                for (int ks = 0; ks < nK; ++ks) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&s_empty[stage]), (uint32_t)((round & 1) ^ 1), &s_abort)) {
+                        if (!s_abort) raise_abort(&s_abort, t.stat, 0x211u);
+                        live = false;
+                        break;
+                    }
+                    const uint32_t full = ptx::smem_u32(&s_full[stage]);
+                    const uint32_t a_dst = ring + (uint32_t)(stage * kStage2Bytes);
+                    const uint32_t b_dst = a_dst + 2u * kABytes;
+                    ptx::mbar_arrive_expect_tx(full, (uint32_t)((it.two ? 2 : 1) * kABytes + it.N * kTileK * 2));
+                    ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, it.m0 * kTileM, full);
+                    if (it.two) ptx::tma_g2s_2d(a_dst + kABytes, &tm_hidden, ks * kTileK, (it.m0 + 1) * kTileM, full);
+                    int r = 0;
+#pragma unroll
+                    for (int b = 4; b >= 0; --b) {
+                        const int rows = 16 << b;
+                        if (it.N - r >= rows) {
+                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK, it.v0 + r, full);
+                            r += rows;
+                        }
+                    }
+                    ++issued;
+                    if (++stage == kStages2) { stage = 0; ++round; }
+                }
+            }
+            if (s_abort) {
+                int first = issued > kStages2 ? issued - kStages2 : 0;
+                for (int q = first; q < issued; ++q)
+                    ptx::mbar_wait(ptx::smem_u32(&s_full[q % kStages2]), (uint32_t)((q / kStages2) & 1), &s_zero);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---- MMA issuer ------------------------------------------------------------------
+        if (lane == 0) {
+            int stage = 0, round = 0;
+            bool live = true;
+            for (int j = 0; live && j < n_items; ++j) {
+                const Item2 it = item2(cta + j * grid, nMG, nM, h.V);
+                if (!ptx::mbar_wait(ptx::smem_u32(&s_acc_empty), (uint32_t)((j & 1) ^ 1), &s_abort)) {
+                    if (!s_abort) raise_abort(&s_abort, t.stat, 0x212u);
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, it.N);
+                for (int ks = 0; ks < nK; ++ks) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&s_full[stage]), (uint32_t)(round & 1), &s_abort)) {
+                        if (!s_abort) raise_abort(&s_abort, t.stat, 0x213u);
+                        live = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_src = ring + (uint32_t)(stage * kStage2Bytes);
+                    const uint64_t a0_desc = ptx::smem_desc_sw128(a_src);
+                    const uint64_t a1_desc = ptx::smem_desc_sw128(a_src + kABytes);
+                    const uint64_t b_desc = ptx::smem_desc_sw128(a_src + 2u * kABytes);
+#pragma unroll
+                    for (int kk = 0; kk < kTileK / 16; ++kk)
+                        ptx::umma_bf16(tmem_base, a0_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc,
+                                       (uint32_t)((ks | kk) != 0));
+                    if (it.two) {
+#pragma unroll
+                        for (int kk = 0; kk < kTileK / 16; ++kk)
+                            ptx::umma_bf16(tmem_base + kTileNMax, a1_desc + (uint64_t)(kk * 2),
+                                           b_desc + (uint64_t)(kk * 2), idesc, (uint32_t)((ks | kk) != 0));
+                    }
+                    ptx::umma_commit(ptx::smem_u32(&s_empty[stage]));
+                    if (++stage == kStages2) { stage = 0; ++round; }
+                }
+                if (live) ptx::umma_commit(ptx::smem_u32(&s_acc_full));
+            }
+            if (n_items > 0) {
+                // everything issued has finished before the tensor memory is released
+                ptx::umma_commit(ptx::smem_u32(&s_done));
+                ptx::mbar_wait(ptx::smem_u32(&s_done), 0u, &s_zero);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---- epilogue: warps 2-5 drain the first accumulator, warps 6-9 the second ---------
+        const int mt = (warp - 2) >> 2;
+        const int quarter = warp & 3;
+        for (int j = 0; j < n_items; ++j) {
+            const Item2 it = item2(cta + j * grid, nMG, nM, h.V);
+            const int row0 = (it.m0 + mt) * kTileM + quarter * 32;
+            const int row = row0 + lane;
+            if (!ptx::mbar_wait(ptx::smem_u32(&s_acc_full), (uint32_t)(j & 1), &s_abort)) {
+                if (lane == 0 && !s_abort) raise_abort(&s_abort, t.stat, 0x214u);
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            Stats st = stats_empty();
+            const bool warp_has_rows = (mt == 0 || it.two) && row0 < R_live;
+            if (warp_has_rows) {
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mt * kTileNMax);
+                for (int c0 = 0; c0 < it.N; c0 += 32) {
+                    float z[32];
+                    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, z);
+                    int n_valid = it.N - c0;
+                    if (h.V - (it.v0 + c0) < n_valid) n_valid = h.V - (it.v0 + c0);
+                    if (n_valid > 32) n_valid = 32;
+                    if (row < R_live && n_valid > 0) fold_chunk(st, z, n_valid, it.v0 + c0);
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&s_acc_empty));
+            if (warp_has_rows && row < R_live)
+                partial_store(P, (size_t)row * n_slices + (size_t)(it.v0 / kTileNMax), st);
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __threadfence();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
 }
 
 // Several M tiles: one warp per row merges that row's per-tile partials; the last block done
@@ -442,6 +694,8 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
     if (dev >= 0 && dev < 64 && !configured[dev]) {
         e = cudaFuncSetAttribute(head_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmem);
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(head_umma2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmem2);
+        if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
     UmmaPlan plan;
@@ -487,7 +741,11 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
     if (!make_map(&tm_h, hid_base, hid_rows, h.d, plan.a_rows)) return cudaErrorInvalidValue;
     for (int b = 0; b < 5; ++b)
         if (!make_map(&tm_w.box[b], h.W, h.V, h.d, 16 << b)) return cudaErrorInvalidValue;
-    head_umma_kernel<<<grid, kThreads, kDynSmem, stream>>>(tm_h, tm_w, hk, t, P, s.ticket, plan);
+    if (plan.nM == 1) {
+        head_umma_kernel<<<grid, kThreads, kDynSmem, stream>>>(tm_h, tm_w, hk, t, P, s.ticket, plan);
+    } else {
+        head_umma2_kernel<<<grid, kThreads2, kDynSmem2, stream>>>(tm_h, tm_w, hk, t, P, plan.nM, plan.n_slices);
+    }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     ++*launched;
