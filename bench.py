@@ -121,13 +121,26 @@ def measured_peaks() -> dict:
             "bf16_tflops_sustained": FALLBACK_BF16_TFLOPS_SUSTAINED, "source": "fallback"}
 
 
+# DRAM bytes (read + write) per launch of the dominant kernel, from the ncu captures summarised under
+# profiles/.  Each entry names the kernel sources it was taken with (sha256 of the files under csrc/):
+# once any of them has changed the counters no longer describe the kernel and the figure reads null.
+NCU_TRAFFIC = {
+}
+
+
 def recorded_traffic(workload: str):
-    """DRAM bytes per launch of the dominant kernel from a committed ncu summary, if there is one."""
-    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
-    try:
-        return json.load(open(path)).get(workload)
-    except Exception:
+    import hashlib
+    ent = NCU_TRAFFIC.get(workload)
+    if not ent:
         return None
+    csrc = os.path.join(ROOT, "paper_2507_17307_b200", "csrc")
+    try:
+        for name, digest in ent["sources"].items():
+            if hashlib.sha256(open(os.path.join(csrc, name), "rb").read()).hexdigest() != digest:
+                return None
+    except OSError:
+        return None
+    return ent["bytes"]
 
 
 # ------------------------------------------------------------------------------------------

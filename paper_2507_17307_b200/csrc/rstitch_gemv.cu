@@ -88,8 +88,11 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
             ptx::mbar_fence_init();
         }
         issued = 0;
-        // hidden rows of this pass -> shared memory (rows past the live count read as zero)
-        for (int i = threadIdx.x; i < RT * d8; i += kThreads) {
+        __syncthreads();                       // barriers ready: the producer may start at once
+        // hidden rows of this pass -> shared memory (rows past the live count read as zero); only
+        // the consumer warps take part, the producer is already streaming W_head
+        if (warp < kConsumerWarps)
+        for (int i = threadIdx.x; i < RT * d8; i += kConsumerWarps * 32) {
             int r = r0 + i / d8, c = i - (i / d8) * d8;
             uint4 v = make_uint4(0, 0, 0, 0);
             if (r < R_live) {
@@ -102,7 +105,6 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
             }
             hid4[i] = v;
         }
-        __syncthreads();
 
         if (warp == kConsumerWarps) {
             // ---- producer: one thread feeds the ring -------------------------------------
@@ -126,6 +128,7 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
             __syncwarp();
         } else {
             // ---- consumers -----------------------------------------------------------------
+            asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");   // hidden rows staged
             Stats st = stats_empty();
             const int my_r = lane & (RT - 1);
             // Slot s always goes to warp (s mod 8), so a warp meets the rounds of a slot in order
