@@ -57,6 +57,11 @@ def _load():
         lib.oracle_compact.restype = None
         lib.oracle_spans.argtypes = [i32p, c.c_int32, i32p, i32p, i32p, i32p]
         lib.oracle_spans.restype = None
+        lib.oracle_latency_ms.argtypes = [f64p, c.c_int32, c.c_int32]
+        lib.oracle_latency_ms.restype = c.c_double
+        lib.oracle_alg1_sequence.argtypes = [c.c_int32, c.c_int32, c.c_double, c.c_int32, i32p, f64p, i32p, f64p,
+                                             f64p, f64p, i32p, i32p, i32p, i32p, i32p, f64p, i32p, i32p, i32p, i32p]
+        lib.oracle_alg1_sequence.restype = None
         _lib = lib
     return _lib
 
@@ -182,3 +187,35 @@ def route(hidden, w_head, tau_nats, row_idx=None, row_seq=None, B=None, seq_len=
     if seq_len is not None:
         out["llm_span"], out["llm_row_off"] = spans(idx, seq_len, kv_len)
     return out
+
+
+def latency_ms(coef, n_inf: int, n_kv: int) -> float:
+    """Eq. 5: a * n_inf * n_kv + b * n_inf^2 + c * n_inf + d, milliseconds; coef = (a, b, c, d)."""
+    cf = np.ascontiguousarray(coef, dtype=np.float64)
+    assert cf.shape == (4,)
+    return float(_load().oracle_latency_ms(_p(cf, ctypes.c_double), int(n_inf), int(n_kv)))
+
+
+def alg1_sequence(prompt_len: int, t_max: int, tau: float, eos_id: int, tok_slm, ent_slm, tok_llm, ent_llm,
+                  coef_slm, coef_llm) -> dict:
+    """Algorithm 1 for one sequence over recorded (token, entropy) streams of the two models."""
+    ts = np.ascontiguousarray(tok_slm, dtype=np.int32)
+    tl = np.ascontiguousarray(tok_llm, dtype=np.int32)
+    es = np.ascontiguousarray(ent_slm, dtype=np.float64)
+    el = np.ascontiguousarray(ent_llm, dtype=np.float64)
+    assert min(ts.size, tl.size, es.size, el.size) >= t_max
+    cs = np.ascontiguousarray(coef_slm, dtype=np.float64)
+    cl = np.ascontiguousarray(coef_llm, dtype=np.float64)
+    y = np.full(max(t_max, 1), -1, dtype=np.int32)
+    i32 = lambda n=1: np.zeros(n, dtype=np.int32)
+    n_out, active, L, ln, kept, steps, done, iters = i32(), i32(), i32(2), i32(), i32(2), i32(2), i32(), i32()
+    lat = np.zeros(1, dtype=np.float64)
+    P = lambda a: _p(a, ctypes.c_int32)
+    D = lambda a: _p(a, ctypes.c_double)
+    _load().oracle_alg1_sequence(int(prompt_len), int(t_max), float(tau), int(eos_id), P(ts), D(es), P(tl), D(el),
+                                 D(cs), D(cl), P(y), P(n_out), P(active), P(L), P(ln), D(lat), P(kept), P(steps),
+                                 P(done), P(iters))
+    n = int(n_out[0])
+    return {"y": y[:n].copy(), "n_out": n, "active": int(active[0]), "L_slm": int(L[0]), "L_llm": int(L[1]),
+            "len": int(ln[0]), "lat_ms": float(lat[0]), "kept_slm": int(kept[0]), "kept_llm": int(kept[1]),
+            "steps_slm": int(steps[0]), "steps_llm": int(steps[1]), "done": int(done[0]), "iters": int(iters[0])}

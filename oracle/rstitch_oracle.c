@@ -199,3 +199,102 @@ void oracle_spans(const int32_t *idx, int32_t count, const int32_t *seq_len,
     }
     row_off[count] = acc;
 }
+
+/* ------------------------------------------------------------------------
+ * Latency estimator and the hybrid decode loop (the steps either side of the
+ * routing decision).
+ * ------------------------------------------------------------------------ */
+
+/*
+ * Eq. 5: estimated latency of one model step that processes n_inf tokens on
+ * top of a KV cache of n_kv entries,
+ *     T = a * n_inf * n_kv + b * n_inf^2 + c * n_inf + d      (milliseconds),
+ * coef = {a, b, c, d} fitted per model (the appendix on latency regression
+ * prints three sets).  A decode step is the same expression at n_inf = 1
+ * (Eq. 6 is read as that special case; its printed right-hand side reuses
+ * the letters c and d for the collapsed coefficients a and b + c + d).
+ */
+double oracle_latency_ms(const double *coef, int32_t n_inf, int32_t n_kv)
+{
+    double ni = (double)n_inf, nk = (double)n_kv;
+    return coef[0] * ni * nk + coef[1] * ni * ni + coef[2] * ni + coef[3];
+}
+
+/*
+ * Algorithm 1 for ONE sequence, written out in the paper's order, with the
+ * two models replaced by recorded streams: at loop index t (0-based here)
+ * the active model m (0 = SLM, 1 = LLM) "generates" token tok[m][t] with
+ * entropy ent[m][t] (nats).  KV caches are represented by their sizes only.
+ *
+ *   L[0] = L[1] = 0, y = [], active = SLM
+ *   for t = 1 .. T_max:
+ *     if L[active] < |x + y|:  prefill on (x + y)[L[active]:]  -> n_inf = |x + y| - L[active],
+ *                              n_kv = L[active];  L[active] <- |x + y| + 1
+ *     else:                    decode -> n_inf = 1, n_kv = L[active];  L[active] <- L[active] + 1
+ *     H_t > tau:   (R-Stitch: switch = true)
+ *        active == SLM: discard y_t, roll KV^SLM back by the one entry just added, active <- LLM, continue
+ *        active == LLM: keep decoding on the LLM
+ *     else if active == LLM: active <- SLM
+ *     append y_t;  stop after appending EOS
+ *
+ * The latency estimate sums Eq. 5 over every model step taken, discarded ones included.
+ *
+ * Outputs: y (capacity y_cap >= t_max), *n_out = |y|, final active, L[2], *len = |x + y|,
+ * *lat_ms, tokens kept from each model, model steps taken by each model, *done = 1 if EOS ended it,
+ * *iters = loop iterations executed.
+ */
+void oracle_alg1_sequence(int32_t prompt_len, int32_t t_max, double tau, int32_t eos_id,
+                          const int32_t *tok_slm, const double *ent_slm,
+                          const int32_t *tok_llm, const double *ent_llm,
+                          const double *coef_slm, const double *coef_llm,
+                          int32_t *y, int32_t *n_out, int32_t *active_out, int32_t *L_out,
+                          int32_t *len_out, double *lat_ms, int32_t *kept, int32_t *steps,
+                          int32_t *done, int32_t *iters)
+{
+    int32_t L[2] = {0, 0};
+    int32_t len = prompt_len;
+    int active = 0;
+    int32_t n = 0;
+    double lat = 0.0;
+    kept[0] = kept[1] = 0;
+    steps[0] = steps[1] = 0;
+    *done = 0;
+    int32_t t = 0;
+    for (t = 0; t < t_max; ++t) {
+        int32_t n_inf, n_kv;
+        if (L[active] < len) {              /* KV cache not up to date: prefill the missing span */
+            n_inf = len - L[active];
+            n_kv = L[active];
+            L[active] = len + 1;
+        } else {                            /* decode */
+            n_inf = 1;
+            n_kv = L[active];
+            L[active] = L[active] + 1;
+        }
+        lat += oracle_latency_ms(active == 0 ? coef_slm : coef_llm, n_inf, n_kv);
+        steps[active] += 1;
+        double H = active == 0 ? ent_slm[t] : ent_llm[t];
+        int32_t yt = active == 0 ? tok_slm[t] : tok_llm[t];
+        const int gen = active;             /* the model that produced y_t */
+        if (oracle_rule(H, tau)) {
+            if (active == 0) {              /* SLM -> LLM: token not kept */
+                L[0] -= 1;                  /* roll back the cache entry this step added */
+                active = 1;
+                continue;
+            }                               /* on the LLM: keep decoding with the LLM */
+        } else if (active == 1) {
+            active = 0;                     /* LLM -> SLM */
+        }
+        kept[gen] += 1;                     /* append y_t */
+        y[n++] = yt;
+        len += 1;
+        if (yt == eos_id) { *done = 1; ++t; break; }
+    }
+    *n_out = n;
+    *active_out = active;
+    L_out[0] = L[0];
+    L_out[1] = L[1];
+    *len_out = len;
+    *lat_ms = lat;
+    *iters = t;
+}

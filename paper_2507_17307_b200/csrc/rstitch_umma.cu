@@ -35,7 +35,7 @@ constexpr int kTileNMax  = 256;
 constexpr int kTileK     = 64;                       // bf16 elements = one 128-byte swizzle row
 constexpr int kABytes    = kTileM * kTileK * 2;      // 16 KB
 constexpr int kBBytes    = kTileNMax * kTileK * 2;   // 32 KB
-constexpr int kRingBytes = 4 * (kABytes + kBBytes);        // 192 KB, cut into as many stages as fit
+constexpr int kRingBytes = 224 * 1024;                     // cut into as many stages as fit
 constexpr int kDynSmem   = kRingBytes + 1024;              // + slack to align the ring to 1024 B
 constexpr int kTmemCols  = 512;
 
