@@ -188,6 +188,66 @@ int rstitch_route_static(const void *hidden /* bf16 [B,d] */, const void *W_head
                          int32_t *tok_out, float *ent_out, uint8_t *route_mask, int32_t *llm_idx,
                          int32_t *llm_count, void *cuda_stream);
 
+/* ---- the steps of Algorithm 1 either side of the decision, batched ------------------------------ */
+
+/* Eq. 5 coefficients of one model (the appendix on latency regression prints three sets), ms:
+ * T(N_inf, N_kv) = a N_inf N_kv + b N_inf^2 + c N_inf + d; a decode step is N_inf = 1 (Eq. 6). */
+typedef struct rstitch_latency_model_s { double a, b, c, d; } rstitch_latency_model_t;
+
+/*
+ * Per-sequence state of the hybrid decode loop (Algorithm 1), a structure of DEVICE arrays owned by
+ * the caller, B entries each unless noted.  The paper runs one sequence; here every sequence of a
+ * batch carries its own copy of the algorithm's variables and all advance one loop iteration per round.
+ *   active   0 = SLM, 1 = LLM          kv_slm, kv_llm   L^SLM, L^LLM (KV-cache sizes)
+ *   seq_len  |x + y|                   n_out            |y|
+ *   done     1 once EOS was appended (a sequence is finished when done = 1 or iters = T_max)
+ *   iters    loop iterations executed
+ *   kept     [2 B]: tokens kept from the SLM at [b], from the LLM at [B + b]
+ *   steps    [2 B]: model steps taken, same layout (discarded SLM steps included)
+ *   lat_ms   float64: latency estimate, the sum of Eq. 5 over every model step taken
+ *   y        [B, y_cap] generated tokens (tokens past y_cap are counted but not stored)
+ */
+typedef struct rstitch_alg1_state_s {
+    int32_t *active, *kv_slm, *kv_llm, *seq_len, *n_out, *done, *iters, *kept, *steps;
+    double  *lat_ms;
+    int32_t *y;
+    int32_t  y_cap;
+} rstitch_alg1_state_t;
+
+/* Algorithm 1's initialisation: both caches empty, y = [], active = SLM, |x + y| = prompt_len[b]. */
+int rstitch_alg1_init(const rstitch_alg1_state_t *s, int B, const int32_t *prompt_len /* device [B] */,
+                      void *cuda_stream);
+
+/*
+ * Before the engine of `model` (0 = SLM, 1 = LLM) runs in this round: the prefill-or-decode test of
+ * Algorithm 1 for every sequence that is not done and whose active model is `model`.
+ *   run_idx [B]      ascending ids of those sequences;  run_count [1] their number
+ *   n_inf [B]        per run entry: tokens to process -- |x + y| - L (prefill of the missing span)
+ *                    when L < |x + y|, else 1 (decode);  n_kv [B]: L before the step
+ *   row_off [B + 1]  exclusive prefix sum of n_inf: the row offsets of the model's batch
+ * Side effects per selected sequence: L <- |x + y| + 1 (prefill) or L + 1 (decode), iters += 1,
+ * steps += 1, lat_ms += Eq. 5 with *latency (a HOST pointer).  A sequence that has used t_max
+ * iterations is no longer selected.  All outputs are device arrays.  One round of the loop is
+ * plan(SLM), plan(LLM), the two model steps and routing decisions, commit(SLM), commit(LLM): both
+ * plans come before either commit (with separate run-list buffers), so that a sequence handed over
+ * by a commit does not run a second time in the same round.
+ */
+int rstitch_alg1_plan(const rstitch_alg1_state_t *s, int B, int model, int t_max,
+                      const rstitch_latency_model_t *latency, int32_t *run_idx, int32_t *run_count,
+                      int32_t *n_inf, int32_t *n_kv, int32_t *row_off, void *cuda_stream);
+
+/*
+ * After the routing decision of that model's batch (Algorithm 1 from "if H_t > tau" to the EOS test):
+ * run entry j (sequence run_idx[j]) has route_mask[j] = (H_t > tau) and the token tok[row], row being
+ * the LAST row of its span (row_off[j + 1] - 1; with row_off = NULL, row = j).
+ *   SLM, mask 1: y_t discarded, L^SLM rolled back by the entry the step added, active <- LLM
+ *   LLM, mask 0: active <- SLM, y_t kept          otherwise: y_t kept, same model
+ * A kept token is appended (y, n_out, seq_len, kept) and ends the sequence if it equals eos_id.
+ */
+int rstitch_alg1_commit(const rstitch_alg1_state_t *s, int B, int model, const int32_t *run_idx,
+                        const int32_t *run_count, const int32_t *row_off, const int32_t *tok,
+                        const uint8_t *route_mask, int32_t eos_id, void *cuda_stream);
+
 /* Handle: owns the scratch memory and the device status word for problems up to the given maxima on
  * the current device.  rstitch_destroy(NULL) is a no-op. */
 int rstitch_create(rstitch_handle_t *out, int maxR, int max_d, int maxV);

@@ -21,6 +21,7 @@ EXPORTS = [
     "rstitch_route", "rstitch_route_ex", "rstitch_route_host", "rstitch_create", "rstitch_destroy",
     "rstitch_workspace_bytes", "rstitch_compact", "rstitch_last_status", "rstitch_status_string",
     "rstitch_path_name", "rstitch_route_static", "rstitch_route_ex_host",
+    "rstitch_alg1_init", "rstitch_alg1_plan", "rstitch_alg1_commit",
 ]
 
 
@@ -52,6 +53,17 @@ class DevStat(C.Structure):
     def as_dict(self):
         return {k: int(getattr(self, k)) for k in
                 ("nan_rows", "bad_row_idx", "bad_span", "timeouts", "timeout_site", "launches")}
+
+
+class LatencyModel(C.Structure):
+    """rstitch_latency_model_t: Eq. 5 coefficients (a, b, c, d), milliseconds."""
+    _fields_ = [("a", C.c_double), ("b", C.c_double), ("c", C.c_double), ("d", C.c_double)]
+
+
+class _Alg1State(C.Structure):
+    _fields_ = [("active", C.c_void_p), ("kv_slm", C.c_void_p), ("kv_llm", C.c_void_p), ("seq_len", C.c_void_p),
+                ("n_out", C.c_void_p), ("done", C.c_void_p), ("iters", C.c_void_p), ("kept", C.c_void_p),
+                ("steps", C.c_void_p), ("lat_ms", C.c_void_p), ("y", C.c_void_p), ("y_cap", C.c_int32)]
 
 
 def library_path() -> str:
@@ -92,6 +104,12 @@ def lib():
         L.rstitch_path_name.restype = C.c_char_p
         L.rstitch_route_static.argtypes = [vp, vp, i, i, i, f, vp, vp, vp, vp, vp, vp]
         L.rstitch_route_static.restype = i
+        L.rstitch_alg1_init.argtypes = [C.POINTER(_Alg1State), i, vp, vp]
+        L.rstitch_alg1_init.restype = i
+        L.rstitch_alg1_plan.argtypes = [C.POINTER(_Alg1State), i, i, i, C.POINTER(LatencyModel), vp, vp, vp, vp, vp, vp]
+        L.rstitch_alg1_plan.restype = i
+        L.rstitch_alg1_commit.argtypes = [C.POINTER(_Alg1State), i, i, vp, vp, vp, vp, vp, C.c_int32, vp]
+        L.rstitch_alg1_commit.restype = i
         _lib = L
     return _lib
 
@@ -354,3 +372,55 @@ def last_status(handle: Optional[Handle] = None) -> dict:
     out = s.as_dict()
     out["status"] = st
     return out
+
+
+class Alg1State:
+    """rstitch_alg1_state_t with its device arrays (torch tensors), plus the per-round run lists."""
+
+    INT_FIELDS = ("active", "kv_slm", "kv_llm", "seq_len", "n_out", "done", "iters")
+
+    def __init__(self, B: int, y_cap: int, device="cuda"):
+        import torch
+        self.B, self.y_cap = int(B), int(y_cap)
+        n = max(self.B, 1)
+        for k in self.INT_FIELDS:
+            setattr(self, k, torch.zeros(n, dtype=torch.int32, device=device))
+        self.kept = torch.zeros(2 * n, dtype=torch.int32, device=device)
+        self.steps = torch.zeros(2 * n, dtype=torch.int32, device=device)
+        self.lat_ms = torch.zeros(n, dtype=torch.float64, device=device)
+        self.y = torch.full((n, self.y_cap), -1, dtype=torch.int32, device=device)
+        # run lists of the two plan calls of a round, one set per model (both plans come before
+        # either commit: a sequence handed over by a commit must not run again in the same round)
+        mk = lambda shape, fill=0: torch.full(shape, fill, dtype=torch.int32, device=device)
+        self.run_idx = [mk((n,), -1), mk((n,), -1)]
+        self.run_count = [mk((1,)), mk((1,))]
+        self.n_inf = [mk((n,)), mk((n,))]
+        self.n_kv = [mk((n,)), mk((n,))]
+        self.row_off = [mk((n + 1,)), mk((n + 1,))]
+        c = _Alg1State()
+        for k in self.INT_FIELDS + ("kept", "steps", "lat_ms", "y"):
+            setattr(c, k, _ptr(getattr(self, k)))
+        c.y_cap = self.y_cap
+        self._c = c
+
+    def init(self, prompt_len, stream=None):
+        st = lib().rstitch_alg1_init(C.byref(self._c), self.B, _ptr(prompt_len), _stream_ptr(stream))
+        if st != 0:
+            raise RstitchError(st, "rstitch_alg1_init")
+
+    def plan(self, model: int, t_max: int, latency: LatencyModel, stream=None):
+        st = lib().rstitch_alg1_plan(C.byref(self._c), self.B, int(model), int(t_max), C.byref(latency),
+                                     _ptr(self.run_idx[model]), _ptr(self.run_count[model]), _ptr(self.n_inf[model]),
+                                     _ptr(self.n_kv[model]), _ptr(self.row_off[model]), _stream_ptr(stream))
+        if st != 0:
+            raise RstitchError(st, "rstitch_alg1_plan")
+
+    def commit(self, model: int, tok, mask, eos_id: int, spans: bool = True, stream=None):
+        """Applies the decision block to the run list of plan(model).  spans=True: tok has one entry
+        per row of the model's batch and a sequence's token is the last row of its span; spans=False:
+        tok has one entry per run entry."""
+        st = lib().rstitch_alg1_commit(C.byref(self._c), self.B, int(model), _ptr(self.run_idx[model]),
+                                       _ptr(self.run_count[model]), _ptr(self.row_off[model]) if spans else None,
+                                       _ptr(tok), _ptr(mask), int(eos_id), _stream_ptr(stream))
+        if st != 0:
+            raise RstitchError(st, "rstitch_alg1_commit")

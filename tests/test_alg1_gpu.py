@@ -1,0 +1,172 @@
+"""GPU parity of the batched Algorithm 1 steps (plan / commit kernels and the Eq. 5 latency sum)
+against the oracle's per-sequence loop: first on recorded (token, entropy) streams, then end to end
+with the routing decision itself producing the tokens and masks on two small LM heads."""
+import os
+
+import numpy as np
+import pytest
+
+import rstitch_inputs as gen
+from parity_util import ENT_TOL, GAP_TOL, to_dev_bf16, to_dev_i32
+
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "latency_coeffs.txt")
+
+
+def coeffs():
+    out = {}
+    for line in open(GOLDEN):
+        if line.strip() and not line.startswith("#"):
+            name, a, b, c, d = line.split()
+            out[name] = (float(a), float(b), float(c), float(d))
+    return out
+
+
+@pytest.fixture(scope="module")
+def rs():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2507_17307_b200 import build
+    build.build_library()
+    import paper_2507_17307_b200 as rs
+    return rs
+
+
+def state_to_host(st):
+    f = lambda t: t.cpu().numpy()
+    B = st.B
+    return {"active": f(st.active)[:B], "kv_slm": f(st.kv_slm)[:B], "kv_llm": f(st.kv_llm)[:B],
+            "seq_len": f(st.seq_len)[:B], "n_out": f(st.n_out)[:B], "done": f(st.done)[:B], "iters": f(st.iters)[:B],
+            "kept": f(st.kept).reshape(2, -1)[:, :B], "steps": f(st.steps).reshape(2, -1)[:, :B],
+            "lat_ms": f(st.lat_ms)[:B], "y": f(st.y)[:B]}
+
+
+def check_against_oracle(oracle, got, b, ref):
+    assert got["y"][b][:ref["n_out"]].tolist() == ref["y"].tolist(), b
+    assert got["n_out"][b] == ref["n_out"] and got["active"][b] == ref["active"]
+    assert (got["kv_slm"][b], got["kv_llm"][b], got["seq_len"][b]) == (ref["L_slm"], ref["L_llm"], ref["len"])
+    assert (got["kept"][0][b], got["kept"][1][b]) == (ref["kept_slm"], ref["kept_llm"])
+    assert (got["steps"][0][b], got["steps"][1][b]) == (ref["steps_slm"], ref["steps_llm"])
+    assert got["iters"][b] == ref["iters"] and got["done"][b] == ref["done"]
+    assert got["lat_ms"][b] == pytest.approx(ref["lat_ms"], rel=1e-12, abs=1e-9)
+
+
+@pytest.mark.parametrize("B,T,seed", [(1, 12, 1), (37, 40, 2), (300, 25, 3), (1000, 9, 4)])
+def test_recorded_streams(rs, oracle, B, T, seed):
+    import torch
+    rng = np.random.default_rng(seed)
+    c = coeffs()
+    lat = [rs.LatencyModel(*c["SLM-1.5B"]), rs.LatencyModel(*c["LLM-7B"])]
+    tau, eos = 0.3, 5
+    prompt = rng.integers(1, 2000, size=B).astype(np.int32)
+    tok = rng.integers(0, 40, size=(2, B, T)).astype(np.int32)              # 5 = EOS turns up now and then
+    ent = rng.choice([0.0, 0.05, tau, np.nextafter(tau, 1.0), 0.9, 6.0], size=(2, B, T))
+    st = rs.Alg1State(B, y_cap=T)
+    st.init(to_dev_i32(prompt))
+    for t in range(T):
+        for m in (0, 1):                       # both plans first: a round is one loop iteration per sequence
+            st.plan(m, T, lat[m])
+        for m in (0, 1):
+            n = int(st.run_count[m].item())
+            idx = st.run_idx[m].cpu().numpy()[:n]
+            n_inf = st.n_inf[m].cpu().numpy()[:n]
+            off = st.row_off[m].cpu().numpy()[:n + 1]
+            assert (np.diff(idx) > 0).all() and (n_inf >= 1).all()
+            assert off[0] == 0 and np.array_equal(np.diff(off), n_inf)
+            rows = np.full(max(int(off[n]), 1), -7, dtype=np.int32)        # only span ends carry tokens
+            if n:
+                rows[off[1:] - 1] = tok[m, idx, t]
+            mask = (ent[m, idx, t] > tau).astype(np.uint8) if n else np.zeros(1, np.uint8)
+            st.commit(m, to_dev_i32(rows), torch.from_numpy(mask).cuda(), eos)
+        if t == 0:
+            assert int(st.run_count[0].item()) == B and int(st.run_count[1].item()) == 0     # decoding starts on the SLM
+    torch.cuda.synchronize()
+    got = state_to_host(st)
+    for b in range(B):
+        ref = oracle.alg1_sequence(int(prompt[b]), T, tau, eos, tok[0, b], ent[0, b], tok[1, b], ent[1, b],
+                                   c["SLM-1.5B"], c["LLM-7B"])
+        check_against_oracle(oracle, got, b, ref)
+    # one more round: T_max iterations are used up, nothing runs and nothing changes
+    for m in (0, 1):
+        st.plan(m, T, lat[m])
+        assert int(st.run_count[m].item()) == 0 and int(st.row_off[m][0].item()) == 0
+    again = state_to_host(st)
+    for k in got:
+        assert np.array_equal(got[k], again[k]), k
+
+
+def test_end_to_end_with_the_routing_decision(rs, oracle):
+    # two small heads; the tokens and masks come from rstitch_route_ex on the model's batch of rows
+    import torch
+    B, T, tau, eos = 16, 10, 0.3, -1
+    c = coeffs()
+    lat = [rs.LatencyModel(*c["SLM-1.5B"]), rs.LatencyModel(*c["LLM-14B"])]
+    handle = rs.Handle(512, 64, 512)
+    for seed in range(20):
+        ws = [gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B * T, d=64, V=512, sigma_w=0.06, seed=8100 + seed,
+                         diffuse_frac=(0.4, 0.4)),
+              gen.scaled(gen.WORKLOADS["c4_llm_b64"], B=B * T, d=64, V=512, sigma_w=0.06, seed=8200 + seed,
+                         diffuse_frac=(0.6, 0.6))]
+        w_bits = [gen.make_w_head(w) for w in ws]
+        hid = [gen.make_hidden(ws[m], w_bits[m], 0)[0].reshape(B, T, 64) for m in (0, 1)]
+        ref_rows = [oracle.route(hid[m].reshape(B * T, 64), w_bits[m], tau) for m in (0, 1)]
+        clear = all((np.abs(r["ent"] - tau) > 4 * ENT_TOL).all() for r in ref_rows)
+        if clear:
+            break
+    assert clear, "no seed kept every stream entropy outside the tolerance band"
+    tok = [r["tok"].reshape(B, T).copy() for r in ref_rows]
+    tie = [(r["gap"] < GAP_TOL).reshape(B, T) for r in ref_rows]      # near-ties: either token is right
+    ent = [r["ent"].reshape(B, T) for r in ref_rows]
+    w_dev = [to_dev_bf16(w) for w in w_bits]
+    rng = np.random.default_rng(77)
+    prompt = rng.integers(1, 9, size=B).astype(np.int32)        # short prompts keep the spans small
+    st = rs.Alg1State(B, y_cap=T)
+    st.init(to_dev_i32(prompt))
+    for t in range(T):
+        for m in (0, 1):
+            st.plan(m, T, lat[m])
+        for m in (0, 1):
+            n = int(st.run_count[m].item())
+            if n == 0:
+                continue
+            idx = st.run_idx[m].cpu().numpy()[:n]
+            off = st.row_off[m].cpu().numpy()[:n + 1]
+            R = int(off[n])
+            rows = gen.f32_to_bf16_bits(rng.standard_normal((R, 64)).astype(np.float32))   # span filler rows
+            rows[off[1:] - 1] = hid[m][idx, t]                                            # span ends: the real step
+            row_seq = np.repeat(np.arange(n, dtype=np.int32), np.diff(off))
+            out = rs.route_ex(handle, to_dev_bf16(rows), w_dev[m], tau, R=R, B=n, row_seq=to_dev_i32(row_seq))
+            st.commit(m, out.tok, out.mask, eos)
+            seen = out.tok.cpu().numpy()[off[1:] - 1]
+            exact = ~tie[m][idx, t]
+            assert np.array_equal(seen[exact], tok[m][idx, t][exact])
+            tok[m][idx, t] = seen              # on a near-tie the stream takes the token the GPU chose
+    torch.cuda.synchronize()
+    got = state_to_host(st)
+    routed_any = False
+    for b in range(B):
+        ref = oracle.alg1_sequence(int(prompt[b]), T, tau, eos, tok[0][b], ent[0][b], tok[1][b], ent[1][b],
+                                   c["SLM-1.5B"], c["LLM-14B"])
+        check_against_oracle(oracle, got, b, ref)
+        routed_any |= ref["steps_llm"] > 0
+    assert routed_any, "the workload never handed a step to the LLM"
+    assert rs.last_status(handle)["timeouts"] == 0
+    handle.destroy()
+
+
+def test_argument_errors(rs):
+    import torch
+    st = rs.Alg1State(4, y_cap=4)
+    lat = rs.LatencyModel(0, 0, 0, 1)
+    L = rs.lib()
+    import ctypes as C
+    assert L.rstitch_alg1_plan(C.byref(st._c), 4, 2, 4, C.byref(lat), None, None, None, None, None, None) == -1
+    p = [st.run_idx[0].data_ptr(), st.run_count[0].data_ptr(), st.n_inf[0].data_ptr(), st.n_kv[0].data_ptr(),
+         st.row_off[0].data_ptr()]
+    assert L.rstitch_alg1_plan(C.byref(st._c), 4, 0, 4, None, *p, None) == -1
+    bad = rs.LatencyModel(float("nan"), 0, 0, 1)
+    assert L.rstitch_alg1_plan(C.byref(st._c), 4, 0, 4, C.byref(bad), *p, None) == -1
+    assert L.rstitch_alg1_init(None, 4, None, None) == -1
+    assert L.rstitch_alg1_commit(C.byref(st._c), 4, 0, None, None, None, None, None, 0, None) == -1
+    torch.cuda.synchronize()
