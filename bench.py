@@ -39,6 +39,10 @@ BENCH_WORKLOADS = {
     "c2_slm_b1": ("c2_slm_b1",), "c3_llm_b1": ("c3_llm_b1",), "c3_llm_b4": ("c3_llm_b4",),
     "c3_llm_b16": ("c3_llm_b16",), "c4_slm_b64": ("c4_slm_b64",),
     "c4_batched": ("c4_slm_b64", "c4_llm_b64"), "c5_catchup": ("c5_catchup",), "c1_tiny": ("c1_tiny",),
+    # one round of the batched hybrid decode loop (Algorithm 1) for 64 sequences, all on the device:
+    # plan(SLM), plan(LLM), SLM head on the sequences decoding on the SLM, LLM head on the others,
+    # commit(SLM), commit(LLM)
+    "alg1_b64": ("c4_slm_b64", "c4_llm_b64"),
 }
 
 
@@ -249,7 +253,7 @@ def main() -> int:
     rs.lib()
 
     heavy = args.workload in ("c5_catchup",)
-    K = args.steps if args.steps is not None else (64 if heavy else (2048 if args.workload == "c4_batched" else 8192))
+    K = args.steps if args.steps is not None else (64 if heavy else (2048 if args.workload in ("c4_batched", "alg1_b64") else 8192))
     Wm = args.warmup if args.warmup is not None else (3 if heavy else 64)
     Wm = max(Wm, 3)
     n_rot = 2 if heavy else 8
@@ -264,6 +268,15 @@ def main() -> int:
         return None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
 
     stream = torch.cuda.current_stream()
+    alg1 = args.workload == "alg1_b64"
+    state = None
+    if alg1:
+        B0 = gen.WORKLOADS[names[0]].B
+        state = rs.Alg1State(B0, y_cap=64, device=dev)
+        state.init(i32_dev(np.random.default_rng(4242 + rank).integers(16, 2048, size=B0)), stream=stream)
+        # fitted coefficients printed in the paper's latency-regression appendix (SLM-1.5B, LLM-7B), ms
+        lat_models = [rs.LatencyModel(0.000021, 0.000231, -0.121046, 27.090929),
+                      rs.LatencyModel(0.000027, 0.000031, -0.045256, 27.040801)]
     handles, prepared = [], [[] for _ in range(n_rot)]
     prev_out = [None] * n_rot
     algo_bytes = 0
@@ -281,7 +294,10 @@ def main() -> int:
             out = rs.RouteOutputs.allocate(R, w.B, dev, spans=True)
             kw = dict(R=R, B=w.B, seq_len=i32_dev(b["seq_len"]), kv_len=i32_dev(b["kv_len"]),
                       row_seq=i32_dev(b["row_seq"]), flags=args.flags, stream=stream)
-            if hi == 1:
+            if alg1:
+                # run entry j of the model's batch reads row j of the pool; the live count is plan's, on device
+                kw = dict(R=w.B, B=w.B, n_rows_dev=state.run_count[hi], flags=args.flags, stream=stream)
+            elif hi == 1:
                 # batched step: the LLM head runs on the subset the SLM head routed, count on device
                 kw.update(row_idx=prev_out[i].llm_idx, n_rows_dev=prev_out[i].llm_count)
             prepared[i].append(rs.PreparedCall(hd, bf16_dev(b["hid"]), w_dev, w.tau_nats, out, **kw))
@@ -293,10 +309,17 @@ def main() -> int:
     decisions_per_step = rows_per_step            # rows decided by the first head of the step
 
     def step(i):
-        for call in prepared[i % n_rot]:
+        calls = prepared[i % n_rot]
+        if alg1:
+            state.plan(0, 1 << 30, lat_models[0], stream=stream)
+            state.plan(1, 1 << 30, lat_models[1], stream=stream)
+        for call in calls:
             st = call.launch()
             if st != 0:
                 raise rs.RstitchError(st, "rstitch_route_ex")
+        if alg1:
+            for m in (0, 1):
+                state.commit(m, calls[m].out.tok, calls[m].out.mask, -1, spans=False, stream=stream)
 
     for i in range(Wm):
         step(i)
@@ -318,7 +341,7 @@ def main() -> int:
         dist.barrier()
     ms = ev0.elapsed_time(ev1)
     stats = [rs.last_status(hd) for hd in handles]
-    launches = sum(st["launches"] for st in stats)
+    launches = sum(st["launches"] for st in stats) + (4 * K if alg1 else 0)
     if any(st["timeouts"] or st["nan_rows"] for st in stats):
         raise SystemExit("device status after the timed region: %s" % stats)
 
@@ -335,7 +358,7 @@ def main() -> int:
 
     host_calls = [[] for _ in range(n_rot)]
     h2d = d2h = 0
-    for hi, h in enumerate(heads):
+    for hi, h in enumerate([] if alg1 else heads):
         w = h["w"]
         for i, b in enumerate(h["batches"]):
             R = b["R"]
@@ -357,7 +380,25 @@ def main() -> int:
                 h2d += b["hid"].shape[0] * w.d * 2 + 4 * n_idx
                 d2h += 8 * R + w.B + 4 * w.B + 4 + 4 * w.B + 4 * (w.B + 1)
 
+    if alg1:
+        # host-fed variant of the same round: both hidden pools come from pinned host memory every round
+        # and the per-sequence token counts go back to the host, with a stream synchronisation
+        pools_host = [[pin(b["hid"].view(np.int16), torch.bfloat16) for b in h["batches"]] for h in heads]
+        pools_dev = [[prepared[i][hi]._keep[1] for i in range(n_rot)] for hi in range(2)]
+        n_out_host = torch.zeros(state.B, dtype=torch.int32).pin_memory()
+        h2d = sum(p[0].numel() * 2 for p in pools_host)
+        d2h = state.B * 4
+
+    def host_step_alg1(i):
+        for hi in range(2):
+            pools_dev[hi][i % n_rot].copy_(pools_host[hi][i % n_rot], non_blocking=True)
+        step(i)
+        n_out_host.copy_(state.n_out[:state.B], non_blocking=True)
+        stream.synchronize()
+
     def host_step(i):
+        if alg1:
+            return host_step_alg1(i)
         calls = host_calls[i % n_rot]
         st = calls[0].launch()
         if st != 0:
@@ -424,8 +465,10 @@ def main() -> int:
         line["e2e"] = {"value": world * decisions_per_step * e2e["steps"] / e2e["seconds"], "unit": UNIT,
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                        "steps": e2e["steps"],
-                       "note": "rstitch_route_ex_host: pinned hidden and index arrays in, tok/ent/mask/llm_idx/"
-                               "llm_count/spans out, stream synchronised every step; W_head resident"}
+                       "note": ("the round's hidden pools copied from pinned host memory, per-sequence token counts "
+                                "copied back, stream synchronised every round; W_head resident") if alg1 else
+                               ("rstitch_route_ex_host: pinned hidden and index arrays in, tok/ent/mask/llm_idx/"
+                                "llm_count/spans out, stream synchronised every step; W_head resident")}
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()

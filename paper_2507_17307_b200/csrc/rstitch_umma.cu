@@ -203,6 +203,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
 
     Schedule sch;
     sch.init(h.V, nM, gridDim.x, blockIdx.x, plan.tiles_per_block);
+    if (R_live == 0) sch.n_items = 0;          // no live rows (device-side count): nothing to stream
 
     if (threadIdx.x == 0) {
         s_abort = 0; s_zero = 0;
@@ -304,9 +305,12 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                 }
                 if (live) ptx::umma_commit(ptx::smem_u32(&s_acc_full[buf]));   // accumulator complete
             }
-            // everything issued has finished before the tensor memory is released
-            ptx::umma_commit(ptx::smem_u32(&s_done));
-            ptx::mbar_wait(ptx::smem_u32(&s_done), 0u, &s_zero);
+            if (sch.n_items > 0) {
+                // everything issued has finished before the tensor memory is released (a commit with
+                // no MMA before it would never arrive)
+                ptx::umma_commit(ptx::smem_u32(&s_done));
+                ptx::mbar_wait(ptx::smem_u32(&s_done), 0u, &s_zero);
+            }
         }
         __syncwarp();
     } else {
@@ -426,7 +430,7 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
     const int nMG = (nM + 1) / 2;
     const int total = ((h.V + kTileNMax - 1) / kTileNMax) * nMG;
     const int cta = blockIdx.x, grid = gridDim.x;
-    const int n_items = cta < total ? (total - cta + grid - 1) / grid : 0;
+    const int n_items = (cta < total && R_live > 0) ? (total - cta + grid - 1) / grid : 0;
 
     if (threadIdx.x == 0) {
         s_abort = 0; s_zero = 0;

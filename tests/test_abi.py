@@ -78,6 +78,35 @@ def test_validation_before_any_cuda_call(rs):
     assert L.rstitch_route_host(None, p, p, 1, 8, 16, 0.5, p, p, p, p, p, None) == -1
 
 
+def test_alg1_validation_before_any_cuda_call(rs):
+    import ctypes as C
+    from paper_2507_17307_b200.binding import _Alg1State, LatencyModel
+    L = rs.lib()
+    one = C.c_int32(0)
+    p = C.addressof(one)
+    st = _Alg1State()
+    lat = LatencyModel(0.0, 0.0, 0.0, 1.0)
+    assert L.rstitch_alg1_init(C.byref(st), 4, p, None) == -1            # state arrays missing
+    for k, _ in _Alg1State._fields_[:-1]:
+        setattr(st, k, p)
+    st.y_cap = 0
+    assert L.rstitch_alg1_init(C.byref(st), 4, p, None) == -1            # no room for tokens
+    st.y_cap = 8
+    assert L.rstitch_alg1_init(C.byref(st), -1, p, None) == -1
+    assert L.rstitch_alg1_init(C.byref(st), 4, None, None) == -1
+    assert L.rstitch_alg1_init(C.byref(st), 0, None, None) == 0          # empty batch: nothing to launch
+    assert L.rstitch_alg1_plan(C.byref(st), 4, 2, 8, C.byref(lat), p, p, p, p, p, None) == -1     # model id
+    assert L.rstitch_alg1_plan(C.byref(st), 4, 0, -1, C.byref(lat), p, p, p, p, p, None) == -1    # T_max
+    assert L.rstitch_alg1_plan(C.byref(st), 4, 0, 8, None, p, p, p, p, p, None) == -1
+    assert L.rstitch_alg1_plan(C.byref(st), 4, 0, 8, C.byref(lat), None, p, p, p, p, None) == -1
+    assert L.rstitch_alg1_plan(C.byref(st), 4, 0, 8, C.byref(LatencyModel(float("inf"), 0, 0, 0)), p, p, p, p, p,
+                               None) == -1
+    assert L.rstitch_alg1_commit(C.byref(st), 4, 0, p, None, None, p, p, 0, None) == -1
+    assert L.rstitch_alg1_commit(C.byref(st), 4, 3, p, p, None, p, p, 0, None) == -1
+    assert L.rstitch_alg1_commit(C.byref(st), 0, 0, None, p, None, None, None, 0, None) == 0
+    assert L.rstitch_route_ex_host(None, None, None) == -1
+
+
 def test_missing_library_fails_loudly(rs, monkeypatch):
     from paper_2507_17307_b200 import binding
     monkeypatch.setattr(binding, "_lib", None)

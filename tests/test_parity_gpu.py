@@ -97,6 +97,10 @@ def test_tensor_core_path_gather_live_count_and_spans(rs, handle, oracle):
     gpu = run_gpu(handle, hid, w_dev, w.tau_nats, row_idx=row_idx, n_rows_dev=live, R=8, flags=rs.PATH_UMMA)
     compare(gpu, ref, w.tau_nats, live, live)
     assert (gpu["tok"][live:8] == -1).all() and (gpu["ent"][live:8] == -1.0).all()
+    # a live count of zero: nothing is evaluated, nothing is routed, every output row stays untouched
+    for flags in (rs.PATH_UMMA, rs.PATH_GEMV):
+        gpu = run_gpu(handle, hid, w_dev, w.tau_nats, row_idx=row_idx, n_rows_dev=0, R=8, flags=flags)
+        assert int(gpu["llm_count"][0]) == 0 and (gpu["tok"][:8] == -1).all() and (gpu["mask"][:8] == 255).all()
     bad = np.array([1, 64, -5, 2], dtype=np.int32)
     gpu = run_gpu(handle, hid, w_dev, w.tau_nats, row_idx=bad, flags=rs.PATH_UMMA)
     ref = oracle.route(hid, w_bits, w.tau_nats, row_idx=np.array([1, 0, 0, 2], dtype=np.int32))
