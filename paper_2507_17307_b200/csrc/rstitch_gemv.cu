@@ -216,7 +216,8 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
     TailArgs ta = t;
     ta.R = R_live;
     if (h.n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
-    tail_finalize_rows(P, n_slices, ta);
+    if (n_slices <= 256 && ta.R <= 2 * (kThreads / 32)) tail_finalize_rows_direct(P, n_slices, ta);
+    else                                                tail_finalize_rows(P, n_slices, ta);
     __syncthreads();
     tail_route(ta, s_tail);
     if (threadIdx.x == 0) *ticket = 0u;

@@ -121,6 +121,60 @@ __device__ inline void tail_finalize_rows(const Partials &P, int n_slices, const
     }
 }
 
+// Finalisation for a handful of rows and at most 256 slices: one warp per row pulls every partial of
+// the row into registers with all loads in flight at once (a single round trip to L2), then merges
+// without a dependent chain: the row maximum M and the greedy token first, then one exponential per
+// partial for the sums.
+__device__ inline void tail_finalize_rows_direct(const Partials &P, int n_slices, const TailArgs &a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int r = warp; r < a.R; r += nwarps) {
+        float m[8], s[8], u[8], bv[8];
+        int bi[8];
+        const size_t base = (size_t)r * n_slices;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int c = lane + 32 * k;
+            const bool in = c < n_slices;
+            const size_t at = base + (in ? c : 0);
+            m[k]  = in ? __ldcg(P.m + at)  : -CUDART_INF_F;
+            s[k]  = in ? __ldcg(P.s + at)  : 0.f;
+            u[k]  = in ? __ldcg(P.u + at)  : 0.f;
+            bv[k] = in ? __ldcg(P.bv + at) : -CUDART_INF_F;
+            bi[k] = in ? __ldcg(P.bi + at) : INT_MAX;
+        }
+        float M = -CUDART_INF_F, best = -CUDART_INF_F;
+        int besti = INT_MAX;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { M = fmaxf(M, m[k]); argmax_take(best, besti, bv[k], bi[k]); }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+            float obv = __shfl_xor_sync(0xffffffffu, best, o);
+            int obi = __shfl_xor_sync(0xffffffffu, besti, o);
+            argmax_take(best, besti, obv, obi);
+        }
+        float ss = 0.f, uu = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (m[k] != -CUDART_INF_F) {
+                const float dm = m[k] - M, e = __expf(dm);
+                ss = fmaf(e, s[k], ss);
+                uu = fmaf(e, fmaf(dm, s[k], u[k]), uu);
+            }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            uu += __shfl_xor_sync(0xffffffffu, uu, o);
+        }
+        if (lane == 0) {
+            Stats t;
+            t.m = M; t.s = ss; t.u = uu; t.bv = best; t.bi = besti;
+            tail_emit_row(t, r, a);
+        }
+    }
+}
+
 // The same finalisation for many rows (tensor-core kernel, up to 128 rows x ~150 slices), where
 // fetching the partials straight from L2 is a chain of dependent round trips.  The partials of a
 // group of rows are first brought into shared memory with five bulk copies (one per statistics
@@ -286,8 +340,45 @@ __device__ inline void tail_compact(const uint8_t *mask, int B, const int32_t *s
     }
 }
 
+// S4-S6 for at most 32 sequences decided row by row: one warp, ballots and shuffles, no block barrier.
+// The entropies were written by this block before its last barrier.
+__device__ inline void tail_route_warp(const TailArgs &a)
+{
+    if (threadIdx.x >= 32) return;
+    const int b = threadIdx.x;
+    const bool in = b < a.B;
+    const bool routed = in && b < a.R && rule(a.ent_out[b], a.tau) != 0;
+    if (in) a.route_mask[b] = routed ? 1 : 0;
+    const unsigned ball = __ballot_sync(0xffffffffu, routed);
+    const int rank = __popc(ball & ((1u << b) - 1u));
+    const bool spans = (a.seq_len != nullptr);
+    int span = 0, incl = 0;
+    if (spans) {
+        if (routed) {
+            span = a.seq_len[b] - a.kv_len[b];
+            if (span < 1) atomicAdd(&a.stat->bad_span, 1u);
+        }
+        incl = span;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (b >= o) incl += v;
+        }
+    }
+    if (routed) {
+        a.llm_idx[rank] = b;
+        if (spans) { a.llm_span[rank] = span; a.llm_row_off[rank] = incl - span; }
+    }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    if (b == 0) {
+        *a.llm_count = __popc(ball);
+        if (spans) a.llm_row_off[__popc(ball)] = total;
+    }
+}
+
 __device__ inline void tail_route(const TailArgs &a, int *smem)
 {
+    if (a.B <= 32 && a.row_seq == nullptr) { tail_route_warp(a); return; }
     tail_mask(a);
     tail_compact(a.route_mask, a.B, a.seq_len, a.kv_len, a.llm_idx, a.llm_count, a.llm_span,
                  a.llm_row_off, a.stat, smem);
