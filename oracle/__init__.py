@@ -57,6 +57,16 @@ def _load():
         lib.oracle_compact.restype = None
         lib.oracle_spans.argtypes = [i32p, c.c_int32, i32p, i32p, i32p, i32p]
         lib.oracle_spans.restype = None
+        u32p = c.POINTER(c.c_uint32)
+        lib.oracle_philox4x32_10.argtypes = [u32p, u32p, u32p]
+        lib.oracle_philox4x32_10.restype = None
+        lib.oracle_sample_uniform.argtypes = [c.c_uint64, c.c_uint64, c.c_uint32, c.c_uint32]
+        lib.oracle_sample_uniform.restype = c.c_double
+        lib.oracle_sample_token.argtypes = [f64p, c.c_int, c.c_double, c.c_uint64, c.c_uint64, c.c_uint32, i32p, f64p]
+        lib.oracle_sample_token.restype = None
+        lib.oracle_sample_rows.argtypes = [u16p, i32p, u16p, c.c_int, c.c_int, c.c_int, c.c_double, c.c_uint64,
+                                           c.c_uint64, i32p, f64p]
+        lib.oracle_sample_rows.restype = None
         lib.oracle_latency_ms.argtypes = [f64p, c.c_int32, c.c_int32]
         lib.oracle_latency_ms.restype = c.c_double
         lib.oracle_alg1_sequence.argtypes = [c.c_int32, c.c_int32, c.c_double, c.c_int32, i32p, f64p, i32p, f64p,
@@ -219,3 +229,46 @@ def alg1_sequence(prompt_len: int, t_max: int, tau: float, eos_id: int, tok_slm,
     return {"y": y[:n].copy(), "n_out": n, "active": int(active[0]), "L_slm": int(L[0]), "L_llm": int(L[1]),
             "len": int(ln[0]), "lat_ms": float(lat[0]), "kept_slm": int(kept[0]), "kept_llm": int(kept[1]),
             "steps_slm": int(steps[0]), "steps_llm": int(steps[1]), "done": int(done[0]), "iters": int(iters[0])}
+
+
+def philox4x32_10(ctr, key):
+    """Philox-4x32-10 (Salmon et al., SC'11): four 32-bit outputs for a 128-bit counter and 64-bit key."""
+    c4 = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k2 = np.ascontiguousarray(key, dtype=np.uint32)
+    assert c4.shape == (4,) and k2.shape == (2,)
+    out = np.zeros(4, dtype=np.uint32)
+    P = lambda a: a.ctypes.data_as(ctypes.POINTER(ctypes.c_uint32))
+    _load().oracle_philox4x32_10(P(c4), P(k2), P(out))
+    return out
+
+
+def sample_uniform(seed: int, draw: int, row: int, v: int) -> float:
+    """The uniform in (0, 1) attached to vocabulary entry v of row `row` at draw number `draw`."""
+    return float(_load().oracle_sample_uniform(int(seed), int(draw), int(row), int(v)))
+
+
+def sample_token(z: np.ndarray, temperature: float, seed: int, draw: int, row: int):
+    """(token, score gap to the runner-up) of the Gumbel-max draw from softmax(z / temperature)."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    tok, gap = ctypes.c_int32(0), ctypes.c_double(0.0)
+    _load().oracle_sample_token(_p(z, ctypes.c_double), z.size, float(temperature), int(seed), int(draw), int(row),
+                                ctypes.byref(tok), ctypes.byref(gap))
+    return int(tok.value), float(gap.value)
+
+
+def sample_rows(hidden, w_head, temperature: float, seed: int, draw: int, row_idx=None):
+    """Sampled token and score gap per row (row r draws with row id r)."""
+    h, w = _u16(hidden), _u16(w_head)
+    V, d = w.shape
+    if row_idx is not None:
+        row_idx = np.ascontiguousarray(row_idx, dtype=np.int32)
+        R = row_idx.size
+    else:
+        R = h.shape[0]
+    tok = np.zeros(R, dtype=np.int32)
+    gap = np.zeros(R, dtype=np.float64)
+    if R:
+        _load().oracle_sample_rows(_p(h, ctypes.c_uint16), _p(row_idx, ctypes.c_int32), _p(w, ctypes.c_uint16), R, d,
+                                   V, float(temperature), int(seed), int(draw), _p(tok, ctypes.c_int32),
+                                   _p(gap, ctypes.c_double))
+    return tok, gap

@@ -298,3 +298,86 @@ void oracle_alg1_sequence(int32_t prompt_len, int32_t t_max, double tau, int32_t
     *lat_ms = lat;
     *iters = t;
 }
+
+/* ------------------------------------------------------------------------
+ * Sampled token (Section 3.1 says y_t is "sampled" from p_t; the sampler is
+ * not specified -- reading: y_t ~ softmax(z / T_s) drawn by the Gumbel-max
+ * construction from a counter-based generator, so that both implementations
+ * draw the same numbers without exchanging them).
+ * ------------------------------------------------------------------------ */
+
+/*
+ * Philox-4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy
+ * as 1, 2, 3", SC'11): ten rounds of
+ *     (c0, c1, c2, c3) <- (hi(M1*c2) ^ c1 ^ k0,  lo(M1*c2),  hi(M0*c0) ^ c3 ^ k1,  lo(M0*c0))
+ * with the key bumped by the Weyl constants (W0, W1) between rounds.
+ */
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) { k0 += W0; k1 += W1; }
+        uint64_t p0 = (uint64_t)M0 * (uint64_t)c0;
+        uint64_t p1 = (uint64_t)M1 * (uint64_t)c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/*
+ * The uniform attached to vocabulary entry v of output row `row` at draw number `draw`:
+ * word (v mod 4) of Philox(counter = (v div 4, row, draw_lo, draw_hi), key = (seed_lo, seed_hi)),
+ * mapped to U = ((x >> 9) + 1/2) / 2^23, an odd multiple of 2^-24 strictly inside (0, 1), which
+ * both float32 and float64 hold exactly.
+ */
+double oracle_sample_uniform(uint64_t seed, uint64_t draw, uint32_t row, uint32_t v)
+{
+    uint32_t ctr[4] = {v >> 2, row, (uint32_t)draw, (uint32_t)(draw >> 32)};
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t out[4];
+    oracle_philox4x32_10(ctr, key, out);
+    uint32_t x = out[v & 3u];
+    return ((double)(x >> 9) + 0.5) / 8388608.0;
+}
+
+/*
+ * Gumbel-max draw: tok = argmax_v ( z[v] / temperature - ln(-ln U_v) ), lowest index on ties;
+ * the argmax of logits plus independent standard Gumbel noise is distributed as softmax(z / T_s).
+ * gap = best score minus the runner-up's.  NaN logits never win; 0 if all are NaN.
+ */
+void oracle_sample_token(const double *z, int V, double temperature, uint64_t seed, uint64_t draw,
+                         uint32_t row, int32_t *tok, double *gap)
+{
+    int best = -1;
+    double best_s = 0.0, second = -INFINITY;
+    for (int v = 0; v < V; ++v) {
+        if (isnan(z[v])) continue;
+        double u = oracle_sample_uniform(seed, draw, row, (uint32_t)v);
+        double s = z[v] / temperature - log(-log(u));
+        if (best < 0) { best = v; best_s = s; }
+        else if (s > best_s) { second = best_s; best = v; best_s = s; }
+        else if (s > second) second = s;
+    }
+    if (best < 0) { *tok = 0; *gap = NAN; return; }
+    *tok = (int32_t)best;
+    *gap = best_s - second;
+}
+
+/* Sampled tokens for R rows (same row addressing as oracle_head_rows); row r draws with row id r. */
+void oracle_sample_rows(const uint16_t *hidden, const int32_t *row_idx, const uint16_t *w_head,
+                        int R, int d, int V, double temperature, uint64_t seed, uint64_t draw,
+                        int32_t *tok, double *gap)
+{
+    double *z = (double *)malloc((size_t)V * sizeof(double));
+    for (int r = 0; r < R; ++r) {
+        size_t src = row_idx ? (size_t)row_idx[r] : (size_t)r;
+        oracle_logits_row(hidden + src * (size_t)d, w_head, d, V, z);
+        oracle_sample_token(z, V, temperature, seed, draw, (uint32_t)r, &tok[r], &gap[r]);
+    }
+    free(z);
+}

@@ -23,6 +23,7 @@ struct rstitch_handle_s {
     int      tile_cap    = 0;
     // staging of rstitch_route_host
     void    *st = nullptr;  size_t st_bytes = 0;     // staging block of the host-buffer calls
+    void    *st_host = nullptr;  size_t st_host_bytes = 0;   // pinned mirror of its output part
     cudaStream_t last_stream = nullptr;
     unsigned launch_count = 0;           // kernels enqueued since the status word was last read
 };
@@ -184,6 +185,7 @@ int rstitch_destroy(rstitch_handle_t h)
 {
     if (!h) return RSTITCH_OK;
     cudaFree(h->ws); cudaFree(h->stat); cudaFree(h->tile_counts); cudaFree(h->st);
+    cudaFreeHost(h->st_host);
     cudaGetLastError();
     delete h;
     return RSTITCH_OK;
@@ -299,9 +301,6 @@ int rstitch_route_ex_host(rstitch_handle_t h, const rstitch_args_t *a, void *cud
     auto h2d = [&](size_t o, const void *src, size_t n) {
         return n == 0 || cudaMemcpyAsync(base + o, src, n, cudaMemcpyHostToDevice, stream) == cudaSuccess;
     };
-    auto d2h = [&](void *dst, size_t o, size_t n) {
-        return n == 0 || cudaMemcpyAsync(dst, base + o, n, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-    };
     bool ok = h2d(o_hid, a->hidden, n_src * a->d * 2);
     if (ok && a->row_idx) ok = h2d(o_ridx, a->row_idx, R * 4);
     if (ok && a->row_seq) ok = h2d(o_rseq, a->row_seq, R * 4);
@@ -325,11 +324,27 @@ int rstitch_route_ex_host(rstitch_handle_t h, const rstitch_args_t *a, void *cud
     st = rstitch_route_ex(h, &dv, cuda_stream);
     if (st != RSTITCH_OK) return st;
 
-    ok = d2h(a->tok_out, o_tok, R * 4) && d2h(a->ent_out, o_ent, R * 4) && d2h(a->llm_idx, o_idx, B * 4) &&
-         d2h(a->llm_count, o_cnt, 4) && d2h(a->route_mask, o_msk, B);
-    if (ok && a->seq_len) ok = d2h(a->llm_span, o_span, B * 4) && d2h(a->llm_row_off, o_roff, (B + 1) * 4);
-    ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+    // the outputs are contiguous in the staging block: one copy into a pinned mirror, then plain
+    // host copies into the caller's buffers (a handful of small device-to-host copies costs more)
+    const size_t out_bytes = off - o_tok;
+    if (out_bytes > h->st_host_bytes) {
+        if (h->st_host) { cudaFreeHost(h->st_host); h->st_host = nullptr; h->st_host_bytes = 0; }
+        if (cudaMallocHost(&h->st_host, out_bytes) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+        h->st_host_bytes = out_bytes;
+    }
+    ok = cudaMemcpyAsync(h->st_host, base + o_tok, out_bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+         cudaStreamSynchronize(stream) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    const char *hb = (const char *)h->st_host - o_tok;
+    std::memcpy(a->tok_out, hb + o_tok, R * 4);
+    std::memcpy(a->ent_out, hb + o_ent, R * 4);
+    std::memcpy(a->llm_idx, hb + o_idx, B * 4);
+    std::memcpy(a->llm_count, hb + o_cnt, 4);
+    std::memcpy(a->route_mask, hb + o_msk, B);
+    if (a->seq_len) {
+        std::memcpy(a->llm_span, hb + o_span, B * 4);
+        std::memcpy(a->llm_row_off, hb + o_roff, (B + 1) * 4);
+    }
     return RSTITCH_OK;
 }
 
