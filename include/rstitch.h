@@ -56,6 +56,7 @@ extern "C" {
 
 /* ---- flags for rstitch_args_t.flags ------------------------------------ */
 #define RSTITCH_TAU_NORMALIZED   0x1u  /* tau is the paper's normalised threshold in [0,1]; multiplied by ln V */
+#define RSTITCH_SAMPLE           0x2u  /* tok_out is sampled from softmax(z / temperature), not the greedy token */
 #define RSTITCH_PATH_GEMV        0x10u /* testing only: force the CUDA-core streaming kernel */
 #define RSTITCH_PATH_UMMA        0x20u /* testing only: force the tcgen05 tensor-core kernel */
 
@@ -87,6 +88,11 @@ typedef struct rstitch_handle_s *rstitch_handle_t;
  *   llm_count   int32 [1]
  *   llm_span    optional int32 [B], llm_row_off optional int32 [B + 1] (required iff seq_len is given).
  *               A routed sequence with span < 1 is counted in devstat.bad_span.
+ *   temperature, seed, draw   with RSTITCH_SAMPLE, tok_out[r] is a draw from softmax(z_r / temperature)
+ *               instead of the greedy token (Section 3.1 says y_t is sampled and names no sampler): the
+ *               Gumbel-max construction tok = argmax_v (z_v / T_s - ln(-ln U_v)), lowest index on ties,
+ *               with U_v word (v mod 4) of Philox-4x32-10(counter = (v div 4, r, draw), key = seed) mapped
+ *               to ((x >> 9) + 1/2) / 2^23.  Entropy, mask and compaction do not depend on the draw.
  *   workspace   optional caller scratch of at least rstitch_workspace_bytes(R, d, V) bytes, 256-byte
  *               aligned; NULL uses the handle's own.  Two calls in flight at once on different
  *               streams must not share a workspace.
@@ -111,6 +117,10 @@ typedef struct rstitch_args_s {
     int32_t       *llm_row_off;
     void          *workspace;
     size_t         workspace_bytes;
+    /* with RSTITCH_SAMPLE (ignored otherwise): */
+    float          temperature;     /* T_s > 0 */
+    uint64_t       seed;            /* generator key */
+    uint64_t       draw;            /* draw number: use a new one for every step */
 } rstitch_args_t;
 
 /* Device status word, accumulated since the handle was created or last read. */

@@ -14,6 +14,7 @@ _LIB_PATH = os.path.join(_HERE, "librstitch.so")
 _lib = None
 
 TAU_NORMALIZED = 0x1
+SAMPLE = 0x2
 PATH_GEMV = 0x10
 PATH_UMMA = 0x20
 
@@ -42,6 +43,7 @@ class _Args(C.Structure):
         ("llm_idx", C.c_void_p), ("llm_count", C.c_void_p),
         ("llm_span", C.c_void_p), ("llm_row_off", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("temperature", C.c_float), ("seed", C.c_uint64), ("draw", C.c_uint64),
     ]
 
 
@@ -205,8 +207,9 @@ def route(hidden, W_head, tau: float, out: Optional[RouteOutputs] = None) -> Rou
 def route_ex(handle: Handle, hidden, W_head, tau: float, *, R: Optional[int] = None,
              B: Optional[int] = None, row_idx=None, row_seq=None, n_rows_dev=None, seq_len=None,
              kv_len=None, flags: int = 0, stream=None, out: Optional[RouteOutputs] = None,
-             workspace=None, check: bool = True):
-    """rstitch_route_ex.  Returns the outputs (or the status when check=False)."""
+             workspace=None, check: bool = True, sample=None):
+    """rstitch_route_ex.  Returns the outputs (or the status when check=False).
+    sample = (temperature, seed, draw) asks for a sampled token (RSTITCH_SAMPLE)."""
     n_src, d = int(hidden.shape[0]), int(hidden.shape[1])
     V = int(W_head.shape[0])
     if R is None:
@@ -226,6 +229,9 @@ def route_ex(handle: Handle, hidden, W_head, tau: float, *, R: Optional[int] = N
     a.llm_span, a.llm_row_off = _ptr(out.llm_span), _ptr(out.llm_row_off)
     if workspace is not None:
         a.workspace, a.workspace_bytes = _ptr(workspace), int(workspace.numel() * workspace.element_size())
+    if sample is not None:
+        a.flags |= SAMPLE
+        a.temperature, a.seed, a.draw = float(sample[0]), int(sample[1]), int(sample[2])
     st = lib().rstitch_route_ex(handle.ptr, C.byref(a), _stream_ptr(stream))
     if not check:
         return st

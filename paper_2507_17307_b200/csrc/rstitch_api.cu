@@ -103,7 +103,10 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a)
     if (a->B < 0 || a->n_src < 0) return RSTITCH_ERR_INVALID_ARG;
     if (!std::isfinite(a->tau)) return RSTITCH_ERR_INVALID_ARG;
     if ((a->flags & RSTITCH_PATH_GEMV) && (a->flags & RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
-    if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
+    if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA))
+        return RSTITCH_ERR_INVALID_ARG;
+    if ((a->flags & RSTITCH_SAMPLE) && !(std::isfinite(a->temperature) && a->temperature > 0.f))
+        return RSTITCH_ERR_INVALID_ARG;
     if (!a->llm_count) return RSTITCH_ERR_INVALID_ARG;
     if (a->row_seq == nullptr && a->B != a->R) return RSTITCH_ERR_INVALID_ARG;
     if (a->row_seq != nullptr && a->n_rows_dev != nullptr) return RSTITCH_ERR_INVALID_ARG;
@@ -210,6 +213,13 @@ int rstitch_route_ex(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_str
     ha.hidden = a->hidden; ha.W = a->W_head; ha.R = a->R; ha.d = a->d; ha.V = a->V;
     ha.n_src = a->n_src > 0 ? a->n_src : a->R;
     ha.row_idx = a->row_idx; ha.n_rows_dev = a->n_rows_dev;
+    ha.sample = SampleArgs{};
+    if (a->flags & RSTITCH_SAMPLE) {
+        ha.sample.on = 1;
+        ha.sample.inv_t = 1.0f / a->temperature;
+        ha.sample.k0 = (uint32_t)a->seed; ha.sample.k1 = (uint32_t)(a->seed >> 32);
+        ha.sample.d0 = (uint32_t)a->draw; ha.sample.d1 = (uint32_t)(a->draw >> 32);
+    }
 
     TailArgs ta;
     ta.R = a->R; ta.B = a->B; ta.V = a->V;

@@ -181,7 +181,9 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
                         float z = acc[v][0];
 #pragma unroll
                         for (int r = 1; r < RT; ++r) z = (my_r == r) ? acc[v][r] : z;
-                        stats_push(st, z, v0 + v);
+                        const float score = h.sample.on ? sample_score(h.sample, z, (uint32_t)(r0 + my_r),
+                                                                       (uint32_t)(v0 + v)) : z;
+                        stats_push(st, z, v0 + v, score);
                     }
                 }
             }

@@ -1,6 +1,7 @@
 // Internal launch interfaces between the C ABI (rstitch_api.cu) and the kernel files.
 #pragma once
 #include "rstitch_tail.cuh"
+#include "rstitch_sample.cuh"
 #include <cuda_runtime.h>
 
 namespace rstitch {
@@ -15,6 +16,7 @@ struct HeadArgs {
     int            R, d, V, n_src;
     const int32_t *row_idx;     // optional gather
     const int32_t *n_rows_dev;  // optional live row count
+    SampleArgs     sample;      // sampled instead of greedy token
 };
 
 struct Scratch {

@@ -84,6 +84,7 @@ extern "C" int rstitch_route_static(const void *hidden, const void *W_head, int 
     HeadArgs ha;
     ha.hidden = hidden; ha.W = W_head; ha.R = B; ha.d = d; ha.V = V; ha.n_src = B;
     ha.row_idx = nullptr; ha.n_rows_dev = nullptr;
+    ha.sample = SampleArgs{};                                   // greedy token
     TailArgs ta;
     ta.R = B; ta.B = B; ta.V = V; ta.tau = tau;
     ta.row_seq = nullptr; ta.seq_len = nullptr; ta.kv_len = nullptr;

@@ -31,10 +31,11 @@ __device__ __forceinline__ void argmax_take(float &bv, int &bi, float v, int i)
     if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
 }
 
-// Add one logit.
-__device__ __forceinline__ void stats_push(Stats &t, float z, int idx)
+// Add one logit; `score` is what the token choice maximises (the logit itself for the greedy
+// token, the logit over the temperature plus Gumbel noise for a sampled one).
+__device__ __forceinline__ void stats_push(Stats &t, float z, int idx, float score)
 {
-    argmax_take(t.bv, t.bi, z, idx);
+    if (z == z) argmax_take(t.bv, t.bi, score, idx);      // a NaN logit never wins
     float mn = fmaxf(t.m, z);                       // fmaxf ignores a NaN operand
     float dm = (t.m == -CUDART_INF_F) ? 0.f : (t.m - mn);
     float a  = __expf(dm);
@@ -44,6 +45,8 @@ __device__ __forceinline__ void stats_push(Stats &t, float z, int idx)
     t.s = a * t.s + e;
     t.m = mn;
 }
+
+__device__ __forceinline__ void stats_push(Stats &t, float z, int idx) { stats_push(t, z, idx, z); }
 
 // Merge b into a (a is the set with the lower vocabulary indices only by convention; the argmax
 // comparison is order-independent).

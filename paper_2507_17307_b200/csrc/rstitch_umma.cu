@@ -97,7 +97,8 @@ __device__ __forceinline__ void raise_abort(volatile int *flag, DevStat *stat, u
 // statistics: one rescale of the running sums per chunk, then one ex2 per logit.  Four independent
 // partial maxima / sums keep the dependent chains short: an epilogue warp has a scheduler to itself,
 // so instruction-level parallelism is all the latency hiding there is.
-__device__ __forceinline__ void fold_chunk_full(Stats &st, const float (&z)[32], int vbase)
+__device__ __forceinline__ void fold_chunk_full(Stats &st, const float (&z)[32], int vbase, const SampleArgs &sa,
+                                                uint32_t row)
 {
     float c0 = fmaxf(z[0], z[4]), c1 = fmaxf(z[1], z[5]), c2 = fmaxf(z[2], z[6]), c3 = fmaxf(z[3], z[7]);
 #pragma unroll
@@ -124,6 +125,20 @@ __device__ __forceinline__ void fold_chunk_full(Stats &st, const float (&z)[32],
     }
     st.s += (s0 + s1) + (s2 + s3);
     st.u += (u0 + u1) + (u2 + u3);
+    if (sa.on) {                              // sampled token: the same for every lane of the warp
+        // vbase is a multiple of 4, so each generator call serves four consecutive columns
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            uint32_t o[4];
+            philox4x32_10((uint32_t)(vbase + i) >> 2, row, sa.d0, sa.d1, sa.k0, sa.k1, o);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float sc = fmaf(z[i + q], sa.inv_t, gumbel_from_bits(o[q]));
+                if (z[i + q] == z[i + q] && sc > st.bv) { st.bv = sc; st.bi = vbase + i + q; }
+            }
+        }
+        return;
+    }
     if (cmax > st.bv) {                       // strictly larger: an earlier chunk keeps a tie
         int idx = 31;
 #pragma unroll
@@ -134,7 +149,8 @@ __device__ __forceinline__ void fold_chunk_full(Stats &st, const float (&z)[32],
 }
 
 // The same for a chunk with fewer than 32 real vocabulary entries (tile tails).
-__device__ __forceinline__ void fold_chunk_tail(Stats &st, const float (&z)[32], int n_valid, int vbase)
+__device__ __forceinline__ void fold_chunk_tail(Stats &st, const float (&z)[32], int n_valid, int vbase,
+                                                const SampleArgs &sa, uint32_t row)
 {
     float cmax = -CUDART_INF_F;
 #pragma unroll
@@ -157,17 +173,19 @@ __device__ __forceinline__ void fold_chunk_tail(Stats &st, const float (&z)[32],
             float e = __expf(dz);
             s += e;
             u = fmaf(e, dz, u);
-            if (z[i] > st.bv) { st.bv = z[i]; st.bi = vbase + i; }   // ascending index: first maximum wins
+            const float sc = sa.on ? sample_score(sa, z[i], row, (uint32_t)(vbase + i)) : z[i];
+            if (z[i] == z[i] && sc > st.bv) { st.bv = sc; st.bi = vbase + i; }   // ascending index: first maximum wins
         }
     }
     st.s += s;
     st.u += u;
 }
 
-__device__ __forceinline__ void fold_chunk(Stats &st, const float (&z)[32], int n_valid, int vbase)
+__device__ __forceinline__ void fold_chunk(Stats &st, const float (&z)[32], int n_valid, int vbase,
+                                           const SampleArgs &sa, uint32_t row)
 {
-    if (n_valid >= 32) fold_chunk_full(st, z, vbase);     // n_valid is the same in every lane
-    else               fold_chunk_tail(st, z, n_valid, vbase);
+    if (n_valid >= 32) fold_chunk_full(st, z, vbase, sa, row);     // n_valid is the same in every lane
+    else               fold_chunk_tail(st, z, n_valid, vbase, sa, row);
 }
 
 // Tensor maps over W_head with boxes of 16, 32, 64, 128 and 256 rows: a tile of N rows (a multiple
@@ -337,7 +355,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                     int n_valid = it.N - c0;
                     if (h.V - (it.v0 + c0) < n_valid) n_valid = h.V - (it.v0 + c0);
                     if (n_valid > 32) n_valid = 32;
-                    if (row < R_live && n_valid > 0) fold_chunk(st, z, n_valid, it.v0 + c0);
+                    if (row < R_live && n_valid > 0) fold_chunk(st, z, n_valid, it.v0 + c0, h.sample, (uint32_t)row);
                 }
             }
             ptx::tc_fence_before_sync();
@@ -562,7 +580,7 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
                     int n_valid = it.N - c0;
                     if (h.V - (it.v0 + c0) < n_valid) n_valid = h.V - (it.v0 + c0);
                     if (n_valid > 32) n_valid = 32;
-                    if (row < R_live && n_valid > 0) fold_chunk(st, z, n_valid, it.v0 + c0);
+                    if (row < R_live && n_valid > 0) fold_chunk(st, z, n_valid, it.v0 + c0, h.sample, (uint32_t)row);
                 }
             }
             ptx::tc_fence_before_sync();

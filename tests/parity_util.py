@@ -28,7 +28,7 @@ def to_dev_i32(a, device="cuda"):
 
 
 def run_gpu(handle, hid_bits, w_dev, tau, *, row_idx=None, row_seq=None, B=None, seq_len=None,
-            kv_len=None, n_rows_dev=None, flags=0, hid_dev=None, R=None):
+            kv_len=None, n_rows_dev=None, flags=0, hid_dev=None, R=None, sample=None):
     """One rstitch_route_ex call; returns numpy outputs (full buffers, canaries included)."""
     import torch
     import paper_2507_17307_b200 as rs
@@ -43,7 +43,7 @@ def run_gpu(handle, hid_bits, w_dev, tau, *, row_idx=None, row_seq=None, B=None,
         kw["seq_len"], kw["kv_len"] = to_dev_i32(seq_len), to_dev_i32(kv_len)
     if n_rows_dev is not None:
         kw["n_rows_dev"] = to_dev_i32([n_rows_dev])
-    out = rs.route_ex(handle, hid_dev, w_dev, tau, B=B, R=R, flags=flags, **kw)
+    out = rs.route_ex(handle, hid_dev, w_dev, tau, B=B, R=R, flags=flags, sample=sample, **kw)
     torch.cuda.synchronize()
     res = {k: getattr(out, k).cpu().numpy() for k in ("tok", "ent", "mask", "llm_idx", "llm_count")}
     if out.llm_span is not None:

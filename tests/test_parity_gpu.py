@@ -370,3 +370,41 @@ def test_standalone_compaction(rs, oracle, B):
             md = torch.full((B,), fill, dtype=torch.uint8, device="cuda")
             idx, cnt = rs.compact(md)
             assert int(cnt.item()) == fill * B
+
+
+# ---- sampled token ---------------------------------------------------------------------------------
+@pytest.mark.parametrize("B,d,V,flags", [
+    (1, 64, 300, "gemv"), (3, 256, 4097, "gemv"), (4, 1536, 9001, "gemv"),
+    (5, 64, 1000, "umma"), (16, 128, 4097, "umma"), (64, 256, 6007, "umma"), (200, 136, 2500, "umma"),
+    (300, 256, 4099, "umma"),
+])
+def test_sampled_token(rs, handle, oracle, B, d, V, flags):
+    flag = rs.PATH_GEMV if flags == "gemv" else rs.PATH_UMMA
+    w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=d, V=V, seed=9900 + B + d + V, sigma_w=0.5 / math.sqrt(d))
+    w_bits = gen.make_w_head(w)
+    w_dev = to_dev_bf16(w_bits)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    ref = oracle.route(hid, w_bits, w.tau_nats)
+    exempt = 0
+    seen = []
+    for T_s, seed, draw in [(1.0, 7, 0), (1.0, 7, 1), (0.6, 2 ** 40 + 5, 2 ** 33 + 9), (2.5, 1, 123456)]:
+        tok, gap = oracle.sample_rows(hid, w_bits, T_s, seed, draw)
+        gpu = run_gpu(handle, hid, w_dev, w.tau_nats, flags=flag, sample=(T_s, seed, draw))
+        ok = (gpu["tok"][:B] == tok) | (gap < 1e-3)
+        assert ok.all(), (T_s, seed, draw, np.flatnonzero(~ok)[:8])
+        exempt += int((gap < 1e-3).sum())
+        # entropy, mask and compaction do not depend on the draw
+        assert np.abs(gpu["ent"][:B] - ref["ent"]).max() <= 2e-3
+        clear = np.abs(ref["ent"] - w.tau_nats) > 2e-3
+        assert np.array_equal(gpu["mask"][:B][clear], ref["mask"][clear])
+        seen.append(gpu["tok"][:B].copy())
+    assert exempt <= max(1, B // 20)
+    if B >= 16:
+        assert not np.array_equal(seen[0], seen[1])          # a new draw number gives new tokens
+        assert not np.array_equal(seen[0], ref["tok"])       # and they are not simply the greedy ones
+    # temperature -> 0 reproduces the greedy token wherever the top-2 logit gap is clear
+    gpu = run_gpu(handle, hid, w_dev, w.tau_nats, flags=flag, sample=(1e-3, 7, 0))
+    clear = ref["gap"] > 0.05
+    assert np.array_equal(gpu["tok"][:B][clear], ref["tok"][clear])
+    assert rs.route_ex(handle, to_dev_bf16(hid), w_dev, 0.3, sample=(0.0, 1, 1), check=False) == -1
+    assert rs.route_ex(handle, to_dev_bf16(hid), w_dev, 0.3, sample=(float("nan"), 1, 1), check=False) == -1
