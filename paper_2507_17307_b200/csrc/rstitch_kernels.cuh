@@ -42,7 +42,7 @@ cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch
 bool        umma_shape_ok(int R, int d, int V);
 size_t      umma_gather_bytes(int R, int d);
 cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
-                             int sm_count, cudaStream_t stream, int *launched);
+                             int sm_count, cudaStream_t stream, int *launched, bool use_pair);
 
 // Upper bound on the partials per row of any kernel for a vocabulary of V rows.
 __host__ __device__ inline size_t max_slices_for(int V)
