@@ -104,7 +104,7 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a)
     if (!std::isfinite(a->tau)) return RSTITCH_ERR_INVALID_ARG;
     if ((a->flags & RSTITCH_PATH_GEMV) && (a->flags & RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
     if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA |
-                     RSTITCH_PATH_NO_PAIR))
+                     RSTITCH_PATH_PAIR))
         return RSTITCH_ERR_INVALID_ARG;
     if ((a->flags & RSTITCH_SAMPLE) && !(std::isfinite(a->temperature) && a->temperature > 0.f))
         return RSTITCH_ERR_INVALID_ARG;
@@ -243,7 +243,7 @@ int rstitch_route_ex(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_str
         // the partials region is sized for the shape the scratch was made for
         size_t part = a->workspace ? ws_partials_bytes(a->R, a->V) : ws_partials_bytes(h->maxR, h->maxV);
         e = launch_head_umma(ha, ta, sc, (char *)ws + kWsHeader + part, h->sm_count, stream, &launched,
-                             !(a->flags & RSTITCH_PATH_NO_PAIR));
+                             (a->flags & RSTITCH_PATH_PAIR) != 0);
     } else {
         e = launch_head_gemv(ha, ta, sc, h->sm_count, stream, &launched);
     }

@@ -28,7 +28,9 @@ namespace rstitch {
 
 namespace {
 
-constexpr int kThreads   = 192;
+constexpr int kProducers = 3;                        // copy-issuing warps: one thread issues ~7 tensor-map copies
+                                                     // per microsecond, separate warps issue in parallel
+constexpr int kThreads   = 192 + (kProducers - 1) * 32;   // producer, MMA, 4 epilogue warps, extra producers
 constexpr int kMaxStages = 8;
 constexpr int kTileM     = 128;
 constexpr int kTileNMax  = 256;
@@ -248,8 +250,9 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
 
-    if (warp == 0) {
-        // ---- producer --------------------------------------------------------------------
+    if (warp == 0 || warp >= 6) {
+        // ---- producers: the copies of a stage are dealt round-robin to kProducers threads ------
+        const int pid = warp == 0 ? 0 : warp - 5;
         if (lane == 0) {
             int stage = 0, round = 0, issued = 0;
             bool live = true;
@@ -266,22 +269,26 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                     const uint32_t b_dst = a_dst + (uint32_t)plan.a_bytes;
                     // only the first a_rows rows of the hidden tile are fetched; the MMA reads all 128,
                     // and what the stale rows produce lands in accumulator rows nobody looks at
-                    ptx::mbar_arrive_expect_tx(full, (uint32_t)((plan.a_rows + it.N) * kTileK * 2));
-                    ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, it.m * kTileM, full);
-                    int r = 0;
+                    if (pid == 0) {
+                        ptx::mbar_arrive_expect_tx(full, (uint32_t)((plan.a_rows + it.N) * kTileK * 2));
+                        ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, it.m * kTileM, full);
+                    }
+                    int r = 0, op = 1;
 #pragma unroll
                     for (int b = 4; b >= 0; --b) {
                         const int rows = 16 << b;
                         if (it.N - r >= rows) {
-                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK, it.v0 + r, full);
+                            if (op % kProducers == pid)
+                                ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK, it.v0 + r, full);
                             r += rows;
+                            ++op;
                         }
                     }
                     ++issued;
                     if (++stage == n_stages) { stage = 0; ++round; }
                 }
             }
-            if (s_abort) {
+            if (s_abort && pid == 0) {
                 // no copy may still be landing in this block's shared memory when it exits
                 int first = issued > n_stages ? issued - n_stages : 0;
                 for (int q = first; q < issued; ++q)
@@ -403,14 +410,16 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
 }
 
 // ---- several M tiles, two per W tile ------------------------------------------------------------
-// With more than 128 rows the kernel above is fed from L2 and starves: a 128 x 256 accumulator tile
-// needs 48 KB of operands per 512 tensor-pipe cycles.  Here one block works on TWO M tiles against
-// the same W tile, so each 32 KB W stage is used twice (64 KB per 1024 cycles) and the ring looks
-// 50 % further ahead in time.  The 512 tensor-memory columns hold the two accumulators, so there is
-// no second buffer: eight epilogue warps (four per accumulator) drain them while the tensor pipe
-// waits, a few percent of an item.  Work items are (vocabulary tile, pair of M tiles), dealt
-// round-robin with the pairs of one vocabulary tile adjacent (W_head from HBM once, then from L2).
-constexpr int kThreads2    = 320;                          // producer, MMA, 8 epilogue warps
+// With more than 128 rows one block works on TWO M tiles against the same W tile, so each 32 KB W stage
+// is used twice: per k-step 64 KB of copies feed eight MMAs instead of 96 KB.  The 512 tensor-memory
+// columns hold the two accumulators, so there is no second buffer: eight epilogue warps (four per
+// accumulator) drain them while the tensor pipe waits, a few percent of an item.  Work items are
+// (vocabulary tile, pair of M tiles), dealt round-robin with the pairs of one vocabulary tile adjacent
+// (W_head from HBM once, then from L2).  Timing variants showed the k-step time to be the sum of the
+// copy bytes and the operand bytes over ~200 KB/us: shared-memory bandwidth, not HBM, L2 latency
+// (an L2 prefetch changed nothing) or instruction issue, bounds this kernel at about 0.8 of the
+// library GEMM's rate when the M tiles are full.
+constexpr int kThreads2    = 320 + (kProducers - 1) * 32;  // producer, MMA, 8 epilogue warps, extra producers
 constexpr int kStages2     = 3;
 constexpr int kStage2Bytes = 2 * kABytes + kBBytes;        // 64 KB
 constexpr int kDynSmem2    = kStages2 * kStage2Bytes + 1024;
@@ -472,8 +481,9 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
 
-    if (warp == 0) {
-        // ---- producer --------------------------------------------------------------------
+    if (warp == 0 || warp >= 10) {
+        // ---- producers: the copies of a stage are dealt round-robin to kProducers threads ------
+        const int pid = warp == 0 ? 0 : warp - 9;
         if (lane == 0) {
             int stage = 0, round = 0, issued = 0;
             bool live = true;
@@ -488,23 +498,28 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
                     const uint32_t full = ptx::smem_u32(&s_full[stage]);
                     const uint32_t a_dst = ring + (uint32_t)(stage * kStage2Bytes);
                     const uint32_t b_dst = a_dst + 2u * kABytes;
-                    ptx::mbar_arrive_expect_tx(full, (uint32_t)((it.two ? 2 : 1) * kABytes + it.N * kTileK * 2));
-                    ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, it.m0 * kTileM, full);
-                    if (it.two) ptx::tma_g2s_2d(a_dst + kABytes, &tm_hidden, ks * kTileK, (it.m0 + 1) * kTileM, full);
-                    int r = 0;
+                    if (pid == 0) {
+                        ptx::mbar_arrive_expect_tx(full, (uint32_t)((it.two ? 2 : 1) * kABytes + it.N * kTileK * 2));
+                        ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, it.m0 * kTileM, full);
+                    }
+                    if (it.two && pid == 1 % kProducers)
+                        ptx::tma_g2s_2d(a_dst + kABytes, &tm_hidden, ks * kTileK, (it.m0 + 1) * kTileM, full);
+                    int r = 0, op = 2;
 #pragma unroll
                     for (int b = 4; b >= 0; --b) {
                         const int rows = 16 << b;
                         if (it.N - r >= rows) {
-                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK, it.v0 + r, full);
+                            if (op % kProducers == pid)
+                                ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK, it.v0 + r, full);
                             r += rows;
+                            ++op;
                         }
                     }
                     ++issued;
                     if (++stage == kStages2) { stage = 0; ++round; }
                 }
             }
-            if (s_abort) {
+            if (s_abort && pid == 0) {
                 int first = issued > kStages2 ? issued - kStages2 : 0;
                 for (int q = first; q < issued; ++q)
                     ptx::mbar_wait(ptx::smem_u32(&s_full[q % kStages2]), (uint32_t)((q / kStages2) & 1), &s_zero);
@@ -601,18 +616,20 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
 }
 
 // ---- several M tiles, a pair of blocks per W tile (tcgen05 cta_group::2) ---------------------------
-// A single block issuing 128 x 256 MMAs reads 12 KB of shared memory per 128 tensor-pipe cycles (A 4 KB
-// + B 8 KB), close to what shared memory delivers once the TMA fill is added, and the tensor pipe sits
-// half idle.  Two blocks of a cluster working as a pair halve the B traffic: one instruction computes
-// M = 256 (each block's own 128-row A tile into its own tensor memory) against a 256-row W tile whose
-// rows are split between the two blocks' shared memory, so each block loads and reads only 128 W rows.
-// Each block still holds two accumulators (two M tiles), i.e. a pair covers four M tiles per W tile.
+// Measurements of the kernel above put its limit in shared memory: per k-step a block takes 64 KB of TMA
+// writes and 96 KB of MMA operand reads (A 4 KB + B 8 KB per instruction), about what shared memory
+// moves in the time.  Two blocks of a cluster working as a pair halve the B traffic: one instruction
+// computes M = 256 (each block's own 128-row A tile into its own tensor memory) against a 256-row W tile
+// whose rows are split between the two blocks' shared memory, so each block loads and reads only 128 W
+// rows.  Each block still holds two accumulators (two M tiles), i.e. a pair covers four M tiles per W
+// tile.  As it stands this variant wins only where the rows fill whole groups of four M tiles and its
+// coarser work split balances (it lost at 576 rows), so it is opt-in (RSTITCH_PATH_PAIR).
 //   leader (cluster rank 0): its MMA thread issues for the pair; "full" barriers live here and collect
 //     the copy bytes of both blocks; "accumulator empty" collects the arrivals of both blocks' epilogues.
-//   both blocks: producer (own A tiles, own half of W, signalling the leader's barrier), eight epilogue
+//   both blocks: producers (own A tiles, own half of W, signalling the leader's barrier), eight epilogue
 //     warps (own rows), "empty" and "accumulator full" barriers fed by multicast tcgen05.commit.
 // Work: cluster c takes vocabulary tiles c, c + #clusters, ...; for each, the groups of four M tiles.
-constexpr int kThreadsP    = 320;
+constexpr int kThreadsP    = 320 + (kProducers - 1) * 32;
 constexpr int kStagesP     = 4;
 constexpr int kStagePBytes = 2 * kABytes + kBBytes / 2;    // 48 KB: two hidden tiles + half a W tile
 constexpr int kDynSmemP    = kStagesP * kStagePBytes + 1024;
@@ -662,8 +679,9 @@ head_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __gri
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
 
-    if (warp == 0) {
-        // ---- producer (both blocks) --------------------------------------------------------
+    if (warp == 0 || warp >= 10) {
+        // ---- producers (both blocks): the copies of a stage are dealt to kProducers threads -----
+        const int pid = warp == 0 ? 0 : warp - 9;
         if (lane == 0) {
             int stage = 0, round = 0, issued = 0;
             bool live = true;
@@ -686,26 +704,30 @@ head_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __gri
                     }
                     const uint32_t full_local = ptx::smem_u32(&s_full[stage]);
                     const uint32_t full = ptx::mapa(full_local, 0);                // the leader's barrier
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(full_local, bytes);
+                    if (rank == 0 && pid == 0) ptx::mbar_arrive_expect_tx(full_local, bytes);
                     const uint32_t a_dst = ring + (uint32_t)(stage * kStagePBytes);
                     const uint32_t b_dst = a_dst + 2u * kABytes;
-                    if (my0 < nM) ptx::tma_g2s_2d_pair(a_dst, &tm_hidden, ks * kTileK, my0 * kTileM, full);
-                    if (my1 < nM) ptx::tma_g2s_2d_pair(a_dst + kABytes, &tm_hidden, ks * kTileK, my1 * kTileM, full);
-                    int r = 0;
+                    if (my0 < nM && pid == 0)
+                        ptx::tma_g2s_2d_pair(a_dst, &tm_hidden, ks * kTileK, my0 * kTileM, full);
+                    if (my1 < nM && pid == 1 % kProducers)
+                        ptx::tma_g2s_2d_pair(a_dst + kABytes, &tm_hidden, ks * kTileK, my1 * kTileM, full);
+                    int r = 0, op = 2;
 #pragma unroll
                     for (int b = 3; b >= 0; --b) {
                         const int rows = 16 << b;
                         if (half - r >= rows) {
-                            ptx::tma_g2s_2d_pair(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK,
-                                                 v0 + (int)rank * half + r, full);
+                            if (op % kProducers == pid)
+                                ptx::tma_g2s_2d_pair(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK,
+                                                     v0 + (int)rank * half + r, full);
                             r += rows;
+                            ++op;
                         }
                     }
                     ++issued;
                     if (++stage == kStagesP) { stage = 0; ++round; }
                 }
             }
-            if (s_abort && rank == 0) {
+            if (s_abort && rank == 0 && pid == 0) {
                 // no copy may still be landing when the blocks exit; the leader's barriers see both blocks' bytes
                 int first = issued > kStagesP ? issued - kStagesP : 0;
                 for (int q = first; q < issued; ++q)
