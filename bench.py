@@ -129,6 +129,15 @@ def measured_peaks() -> dict:
 # profiles/.  Each entry names the kernel sources it was taken with (sha256 of the files under csrc/):
 # once any of them has changed the counters no longer describe the kernel and the figure reads null.
 NCU_TRAFFIC = {
+    "c2_slm_b1":
+    {"bytes": 470720256, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
+     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "9b926ebd1d559dc9a04ae4c80c5207d485f26a73d6e19ed5c004030677832df1", "rstitch_tail.cuh": "213850b579815c8438459e1885c78989dfc75244b76a8d4197f62012dd3a097f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "248e633f5dbc3c719b09cc1f421c09ead4e2f15e7339d91091252fd0c3e72569"}},
+    "c4_slm_b64":
+    {"bytes": 471161344, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
+     "sources": {"rstitch_umma.cu": "49c9d68e6d65fcbfe0dd5965a2fe5c9e3b6c4962d5bcbed311c70afbe593b9b5", "rstitch_kernels.cuh": "9b926ebd1d559dc9a04ae4c80c5207d485f26a73d6e19ed5c004030677832df1", "rstitch_tail.cuh": "213850b579815c8438459e1885c78989dfc75244b76a8d4197f62012dd3a097f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "248e633f5dbc3c719b09cc1f421c09ead4e2f15e7339d91091252fd0c3e72569"}},
+    "c5_catchup":
+    {"bytes": 1672081912, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
+     "sources": {"rstitch_umma.cu": "49c9d68e6d65fcbfe0dd5965a2fe5c9e3b6c4962d5bcbed311c70afbe593b9b5", "rstitch_kernels.cuh": "9b926ebd1d559dc9a04ae4c80c5207d485f26a73d6e19ed5c004030677832df1", "rstitch_tail.cuh": "213850b579815c8438459e1885c78989dfc75244b76a8d4197f62012dd3a097f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "248e633f5dbc3c719b09cc1f421c09ead4e2f15e7339d91091252fd0c3e72569"}},
 }
 
 
@@ -222,6 +231,8 @@ def main() -> int:
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="rstitch_args_t.flags (testing)")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture one rotation of steps into a CUDA graph and time its replays")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -324,24 +335,56 @@ def main() -> int:
     for i in range(Wm):
         step(i)
     torch.cuda.synchronize()
-    for hd in handles:
-        rs.last_status(hd)                       # clears the launch counters
+    warm_launches = sum(rs.last_status(hd)["launches"] for hd in handles)     # also clears the counters
+    launches_per_step = warm_launches / float(Wm) + (4 if alg1 else 0)
 
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
+    graph = None
+    if args.graph:
+        # the step loop has no host synchronisation, so a whole rotation of steps records into one graph
+        K = max(n_rot, (K // n_rot) * n_rot)
+        cap_stream = torch.cuda.Stream()
+        cap_stream.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(cap_stream):
+            saved = stream
+            stream = cap_stream
+            for calls in prepared:
+                for c in calls:
+                    c._stream = int(cap_stream.cuda_stream)
+            with torch.cuda.graph(graph, stream=cap_stream):
+                for i in range(n_rot):
+                    step(i)
+            stream = saved
+            for calls in prepared:
+                for c in calls:
+                    c._stream = int(saved.cuda_stream) or None
+        torch.cuda.synchronize()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        for hd in handles:
+            rs.last_status(hd)
     with ClockSampler(visible_gpu_index(local_rank)) as clocks:
-        ev0.record(stream)
-        for i in range(K):
-            step(i)
-        ev1.record(stream)
+        ev0.record(torch.cuda.current_stream())
+        if graph is not None:
+            for _ in range(K // n_rot):
+                graph.replay()
+        else:
+            for i in range(K):
+                step(i)
+        ev1.record(torch.cuda.current_stream())
         torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     ms = ev0.elapsed_time(ev1)
     stats = [rs.last_status(hd) for hd in handles]
     launches = sum(st["launches"] for st in stats) + (4 * K if alg1 else 0)
+    if graph is not None:
+        launches = int(round(K * launches_per_step))      # replayed kernels are not counted by the handles
     if any(st["timeouts"] or st["nan_rows"] for st in stats):
         raise SystemExit("device status after the timed region: %s" % stats)
 
@@ -458,7 +501,8 @@ def main() -> int:
                        "path": [rs.path_name(int(rows_per_step), h["w"].d, h["w"].V, args.flags) for h in heads],
                        "l2": "inputs larger than L2: each step streams the whole W_head (%.0f MB); "
                              "hidden rotates over %d buffers" % (algo_bytes / 1e6, n_rot),
-                       "parallelism": "dp%d (rows sharded, head replicated, no collective)" % world},
+                       "parallelism": "dp%d (rows sharded, head replicated, no collective)" % world,
+                       "cuda_graph": bool(args.graph)},
             "roofline": roof, "clocks": clocks.summary(), "gpu_launches": launches,
             "algorithmic_bytes_per_step": algo_bytes, "flops_per_step": flops,
         }

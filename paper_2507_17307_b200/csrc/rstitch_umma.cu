@@ -28,8 +28,10 @@ namespace rstitch {
 
 namespace {
 
-constexpr int kProducers = 3;                        // copy-issuing warps: one thread issues ~7 tensor-map copies
-                                                     // per microsecond, separate warps issue in parallel
+constexpr int kProducers = 1;                        // copy-issuing warps.  One thread issues ~7 tensor-map copies per
+                                                     // microsecond and separate warps issue in parallel (a probe reached
+                                                     // 19/us with four), but these kernels need at most ~6/us and measured
+                                                     // the same with 1, 2 and 3; the dealing code below stays general
 constexpr int kThreads   = 192 + (kProducers - 1) * 32;   // producer, MMA, 4 epilogue warps, extra producers
 constexpr int kMaxStages = 8;
 constexpr int kTileM     = 128;

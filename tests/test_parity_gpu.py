@@ -415,3 +415,40 @@ def test_sampled_token(rs, handle, oracle, B, d, V, flags):
     assert np.array_equal(gpu["tok"][:B][clear], ref["tok"][clear])
     assert rs.route_ex(handle, to_dev_bf16(hid), w_dev, 0.3, sample=(0.0, 1, 1), check=False) == -1
     assert rs.route_ex(handle, to_dev_bf16(hid), w_dev, 0.3, sample=(float("nan"), 1, 1), check=False) == -1
+
+
+def test_step_loop_replays_from_a_cuda_graph(rs, handle, oracle):
+    # a chain of calls with no host synchronisation (SLM head, then the LLM head on the routed subset with
+    # the count on the device) records into a CUDA graph; replays give what the direct calls gave
+    import torch
+    ws = gen.scaled(gen.WORKLOADS["c4_slm_b64"], V=3000, d=512, B=64)
+    wl = gen.scaled(gen.WORKLOADS["c4_llm_b64"], V=2600, d=640, B=64)
+    s_bits, l_bits = gen.make_w_head(ws), gen.make_w_head(wl)
+    s_dev, l_dev = to_dev_bf16(s_bits), to_dev_bf16(l_bits)
+    hs = to_dev_bf16(gen.make_hidden(ws, s_bits, 0)[0])
+    hl = to_dev_bf16(gen.make_hidden(wl, l_bits, 0)[0])
+    h2 = rs.Handle(64, 640, 2600)
+    side = torch.cuda.Stream()
+    out_s = rs.RouteOutputs.allocate(64, 64, hs.device)
+    out_l = rs.RouteOutputs.allocate(64, 64, hs.device)
+    c1 = rs.PreparedCall(handle, hs, s_dev, ws.tau_nats, out_s, stream=side)
+    c2 = rs.PreparedCall(h2, hl, l_dev, wl.tau_nats, out_l, R=64, B=64, row_idx=out_s.llm_idx,
+                         n_rows_dev=out_s.llm_count, stream=side)
+    with torch.cuda.stream(side):
+        assert c1.launch() == 0 and c2.launch() == 0            # first calls outside the capture
+    side.synchronize()
+    want = [t.clone() for t in (out_s.tok, out_s.ent, out_s.mask, out_s.llm_count, out_l.tok, out_l.ent, out_l.llm_count)]
+    cnt = int(out_s.llm_count.item())
+    assert 0 < cnt < 64
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        assert c1.launch() == 0 and c2.launch() == 0
+    for t in (out_s.tok, out_s.ent, out_l.tok, out_l.ent):
+        t.fill_(-1)
+    g.replay()
+    torch.cuda.synchronize()
+    got = [out_s.tok, out_s.ent, out_s.mask, out_s.llm_count, out_l.tok, out_l.ent, out_l.llm_count]
+    for i, (a, b) in enumerate(zip(want, got)):
+        n = cnt if i in (4, 5) else a.shape[0]          # the LLM head wrote only the routed rows
+        assert torch.equal(a[:n], b[:n]), i
+    h2.destroy()
