@@ -203,6 +203,7 @@ struct UmmaPlan {
     int a_rows;            // hidden rows fetched per k-step (the MMA still reads 128)
     int n_stages, a_bytes, stage_bytes;
     int tiles_per_block;   // one M tile only
+    int m64;               // one M tile only: at most 64 rows, issue M = 64 instructions
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -311,7 +312,9 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, it.N);
+                // with at most 64 rows an M = 64 instruction does half the tensor work and reads half the
+                // hidden tile; its 64 accumulator rows sit in lanes 0-15 of each 32-lane quarter
+                const uint32_t idesc = ptx::umma_idesc_bf16(plan.m64 ? 64 : kTileM, it.N);
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * kTileNMax;
                 for (int ks = 0; ks < nK; ++ks) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&s_full[stage]), (uint32_t)(round & 1), &s_abort)) {
@@ -343,7 +346,10 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     } else {
         // ---- epilogue --------------------------------------------------------------------
         const int quarter = warp & 3;                        // the TMEM lanes this warp may read
-        const int row_in_tile = quarter * 32 + lane;
+        // M = 128: accumulator row i is lane i.  M = 64: row i is lane 32 (i / 16) + i % 16.
+        const int rows_per_quarter = plan.m64 ? 16 : 32;
+        const int row_in_tile = quarter * rows_per_quarter + lane;
+        const bool lane_has_row = lane < rows_per_quarter;
         Stats st = stats_empty();
         for (int j = 0; j < sch.n_items; ++j) {
             const Item it = sch.item(j);
@@ -354,7 +360,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                 break;
             }
             ptx::tc_fence_after_sync();
-            const bool warp_has_rows = (it.m * kTileM + quarter * 32) < R_live;
+            const bool warp_has_rows = (it.m * kTileM + quarter * rows_per_quarter) < R_live;
             if (nM > 1) st = stats_empty();
             if (warp_has_rows) {
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kTileNMax;
@@ -364,16 +370,17 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                     int n_valid = it.N - c0;
                     if (h.V - (it.v0 + c0) < n_valid) n_valid = h.V - (it.v0 + c0);
                     if (n_valid > 32) n_valid = 32;
-                    if (row < R_live && n_valid > 0) fold_chunk(st, z, n_valid, it.v0 + c0, h.sample, (uint32_t)row);
+                    if (lane_has_row && row < R_live && n_valid > 0)
+                        fold_chunk(st, z, n_valid, it.v0 + c0, h.sample, (uint32_t)row);
                 }
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&s_acc_empty[buf]));
-            if (nM > 1 && row < R_live)
+            if (nM > 1 && lane_has_row && row < R_live)
                 partial_store(P, (size_t)row * n_slices + (size_t)(it.v0 / kTileNMax), st);
         }
-        if (nM == 1 && row_in_tile < R_live)
+        if (nM == 1 && lane_has_row && row_in_tile < R_live)
             partial_store(P, (size_t)row_in_tile * n_slices + blockIdx.x, st);
     }
 
@@ -427,6 +434,13 @@ constexpr int kStage2Bytes = 2 * kABytes + kBBytes;        // 64 KB
 constexpr int kDynSmem2    = kStages2 * kStage2Bytes + 1024;
 
 struct Item2 { int v0, N, m0, two; };
+
+// An M tile that holds at most 64 of the R rows (the last, partly filled one).
+__device__ __forceinline__ bool tile_is_small(int tile, int R)
+{
+    const int rows = R - tile * kTileM;
+    return rows > 0 && rows <= 64;
+}
 
 __device__ __forceinline__ Item2 item2(int q, int nMG, int nM, int V)
 {
@@ -540,7 +554,9 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
                     break;
                 }
                 ptx::tc_fence_after_sync();
-                const uint32_t idesc = ptx::umma_idesc_bf16(kTileM, it.N);
+                // an M tile with at most 64 rows (the last one) takes M = 64 instructions
+                const uint32_t idesc0 = ptx::umma_idesc_bf16(tile_is_small(it.m0, h.R) ? 64 : kTileM, it.N);
+                const uint32_t idesc1 = ptx::umma_idesc_bf16(tile_is_small(it.m0 + 1, h.R) ? 64 : kTileM, it.N);
                 for (int ks = 0; ks < nK; ++ks) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&s_full[stage]), (uint32_t)(round & 1), &s_abort)) {
                         if (!s_abort) raise_abort(&s_abort, t.stat, 0x213u);
@@ -554,13 +570,13 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
                     const uint64_t b_desc = ptx::smem_desc_sw128(a_src + 2u * kABytes);
 #pragma unroll
                     for (int kk = 0; kk < kTileK / 16; ++kk)
-                        ptx::umma_bf16(tmem_base, a0_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc,
+                        ptx::umma_bf16(tmem_base, a0_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), idesc0,
                                        (uint32_t)((ks | kk) != 0));
                     if (it.two) {
 #pragma unroll
                         for (int kk = 0; kk < kTileK / 16; ++kk)
                             ptx::umma_bf16(tmem_base + kTileNMax, a1_desc + (uint64_t)(kk * 2),
-                                           b_desc + (uint64_t)(kk * 2), idesc, (uint32_t)((ks | kk) != 0));
+                                           b_desc + (uint64_t)(kk * 2), idesc1, (uint32_t)((ks | kk) != 0));
                     }
                     ptx::umma_commit(ptx::smem_u32(&s_empty[stage]));
                     if (++stage == kStages2) { stage = 0; ++round; }
@@ -580,8 +596,10 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
         const int quarter = warp & 3;
         for (int j = 0; j < n_items; ++j) {
             const Item2 it = item2(cta + j * grid, nMG, nM, h.V);
-            const int row0 = (it.m0 + mt) * kTileM + quarter * 32;
+            const int rows_per_quarter = tile_is_small(it.m0 + mt, h.R) ? 16 : 32;     // M = 64: 16 rows per quarter
+            const int row0 = (it.m0 + mt) * kTileM + quarter * rows_per_quarter;
             const int row = row0 + lane;
+            const bool lane_has_row = lane < rows_per_quarter;
             if (!ptx::mbar_wait(ptx::smem_u32(&s_acc_full), (uint32_t)(j & 1), &s_abort)) {
                 if (lane == 0 && !s_abort) raise_abort(&s_abort, t.stat, 0x214u);
                 break;
@@ -597,13 +615,14 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
                     int n_valid = it.N - c0;
                     if (h.V - (it.v0 + c0) < n_valid) n_valid = h.V - (it.v0 + c0);
                     if (n_valid > 32) n_valid = 32;
-                    if (row < R_live && n_valid > 0) fold_chunk(st, z, n_valid, it.v0 + c0, h.sample, (uint32_t)row);
+                    if (lane_has_row && row < R_live && n_valid > 0)
+                        fold_chunk(st, z, n_valid, it.v0 + c0, h.sample, (uint32_t)row);
                 }
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&s_acc_empty));
-            if (warp_has_rows && row < R_live)
+            if (warp_has_rows && lane_has_row && row < R_live)
                 partial_store(P, (size_t)row * n_slices + (size_t)(it.v0 / kTileNMax), st);
         }
     }
@@ -974,6 +993,7 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
     // 128 hidden rows from the stage's start whatever was fetched, so the last stage keeps that
     // much room inside the ring.
     plan.a_rows = plan.nM == 1 ? ((h.R + 7) / 8) * 8 : kTileM;
+    plan.m64 = (plan.nM == 1 && h.R <= 64) ? 1 : 0;
     plan.a_bytes = ((plan.a_rows * kTileK * 2 + 1023) / 1024) * 1024;
     plan.stage_bytes = plan.a_bytes + n_max * kTileK * 2;
     plan.n_stages = (kRingBytes - (kABytes - plan.a_bytes)) / plan.stage_bytes;
