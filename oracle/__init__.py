@@ -67,6 +67,10 @@ def _load():
         lib.oracle_sample_rows.argtypes = [u16p, i32p, u16p, c.c_int, c.c_int, c.c_int, c.c_double, c.c_uint64,
                                            c.c_uint64, i32p, f64p]
         lib.oracle_sample_rows.restype = None
+        f32p = c.POINTER(c.c_float)
+        lib.oracle_router_rows.argtypes = [u16p, i32p, c.c_int, c.c_int, c.c_int, c.c_int, c.c_int] + [f32p] * 10 + \
+                                          [f64p, u8p]
+        lib.oracle_router_rows.restype = None
         lib.oracle_latency_ms.argtypes = [f64p, c.c_int32, c.c_int32]
         lib.oracle_latency_ms.restype = c.c_double
         lib.oracle_alg1_sequence.argtypes = [c.c_int32, c.c_int32, c.c_double, c.c_int32, i32p, f64p, i32p, f64p,
@@ -272,3 +276,29 @@ def sample_rows(hidden, w_head, temperature: float, seed: int, draw: int, row_id
                                    V, float(temperature), int(seed), int(draw), _p(tok, ctypes.c_int32),
                                    _p(gap, ctypes.c_double))
     return tok, gap
+
+
+ROUTER_KEYS = ("W_in", "b_in", "W1", "b1", "W2", "b2", "ln_g", "ln_b", "W_out", "b_out")
+
+
+def router_rows(hidden, weights: dict, row_idx=None):
+    """R-Stitch+ router forward: (logits float64 [R, 2], switch uint8 [R]).  weights holds float32 arrays
+    W_in [h, d], b_in [h], W1 [L, ff, h], b1 [L, ff], W2 [L, h, ff], b2 [L, h], ln_g [h], ln_b [h],
+    W_out [2, h], b_out [2]."""
+    hb = _u16(hidden)
+    w = {k: np.ascontiguousarray(weights[k], dtype=np.float32) for k in ROUTER_KEYS}
+    h, d = w["W_in"].shape
+    L, ff, _ = w["W1"].shape
+    assert hb.shape[1] == d and w["W2"].shape == (L, h, ff) and w["W_out"].shape == (2, h)
+    if row_idx is not None:
+        row_idx = np.ascontiguousarray(row_idx, dtype=np.int32)
+        R = row_idx.size
+    else:
+        R = hb.shape[0]
+    logits = np.zeros((max(R, 1), 2), dtype=np.float64)
+    sw = np.zeros(max(R, 1), dtype=np.uint8)
+    if R:
+        _load().oracle_router_rows(_p(hb, ctypes.c_uint16), _p(row_idx, ctypes.c_int32), R, d, h, ff, L,
+                                   *[_p(w[k], ctypes.c_float) for k in ROUTER_KEYS],
+                                   _p(logits, ctypes.c_double), _p(sw, ctypes.c_uint8))
+    return logits[:R], sw[:R]

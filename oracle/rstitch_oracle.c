@@ -381,3 +381,74 @@ void oracle_sample_rows(const uint16_t *hidden, const int32_t *row_idx, const ui
     }
     free(z);
 }
+
+/* ------------------------------------------------------------------------
+ * R-Stitch+ router forward (the "Architecture and Overhead of Router" appendix:
+ * a small feed-forward network on the hidden state -- 6 FFN blocks with GELU and
+ * residual connections, then normalisation, then a two-head linear layer).  The
+ * paper gives neither widths nor weights; the reading taken is
+ *     x0 = W_in s + b_in                                   (d -> h)
+ *     x_{l+1} = x_l + W2_l GELU(W1_l x_l + b1_l) + b2_l      (h -> ff -> h), l = 0 .. n_blocks-1
+ *     y = LayerNorm(x) * g + beta                           (eps = 1e-5, biased variance)
+ *     logits = W_out y + b_out                              (h -> 2: SLM, LLM)
+ * with the exact (erf) GELU.  Algorithm 1: switch = (argmax_a pi(a | s_t) == LLM).
+ * ------------------------------------------------------------------------ */
+static double gelu_exact(double x) { return 0.5 * x * (1.0 + erf(x / sqrt(2.0))); }
+
+/* hidden: bf16 bits [d].  All weights fp32, row-major as named above.  logits[2]. */
+void oracle_router_row(const uint16_t *hidden, int d, int h, int ff, int n_blocks,
+                       const float *W_in, const float *b_in, const float *W1, const float *b1,
+                       const float *W2, const float *b2, const float *ln_g, const float *ln_b,
+                       const float *W_out, const float *b_out, double *logits)
+{
+    double *x = (double *)malloc((size_t)h * sizeof(double));
+    double *t = (double *)malloc((size_t)ff * sizeof(double));
+    for (int i = 0; i < h; ++i) {
+        double acc = (double)b_in[i];
+        for (int k = 0; k < d; ++k) acc += (double)W_in[(size_t)i * d + k] * bf16_to_double(hidden[k]);
+        x[i] = acc;
+    }
+    for (int l = 0; l < n_blocks; ++l) {
+        const float *w1 = W1 + (size_t)l * ff * h, *w2 = W2 + (size_t)l * h * ff;
+        for (int j = 0; j < ff; ++j) {
+            double acc = (double)b1[(size_t)l * ff + j];
+            for (int i = 0; i < h; ++i) acc += (double)w1[(size_t)j * h + i] * x[i];
+            t[j] = gelu_exact(acc);
+        }
+        for (int i = 0; i < h; ++i) {
+            double acc = (double)b2[(size_t)l * h + i];
+            for (int j = 0; j < ff; ++j) acc += (double)w2[(size_t)i * ff + j] * t[j];
+            x[i] += acc;                                    /* residual */
+        }
+    }
+    double mean = 0.0, var = 0.0;
+    for (int i = 0; i < h; ++i) mean += x[i];
+    mean /= (double)h;
+    for (int i = 0; i < h; ++i) var += (x[i] - mean) * (x[i] - mean);
+    var /= (double)h;
+    const double inv = 1.0 / sqrt(var + 1e-5);
+    for (int a = 0; a < 2; ++a) {
+        double acc = (double)b_out[a];
+        for (int i = 0; i < h; ++i)
+            acc += (double)W_out[(size_t)a * h + i] * ((x[i] - mean) * inv * (double)ln_g[i] + (double)ln_b[i]);
+        logits[a] = acc;
+    }
+    free(x);
+    free(t);
+}
+
+/* R rows (row r reads hidden[row_idx[r]] when row_idx != NULL); logits [R, 2];
+ * switch_llm[r] = 1 iff the LLM logit is strictly larger (a tie keeps the SLM). */
+void oracle_router_rows(const uint16_t *hidden, const int32_t *row_idx, int R, int d, int h, int ff,
+                        int n_blocks, const float *W_in, const float *b_in, const float *W1,
+                        const float *b1, const float *W2, const float *b2, const float *ln_g,
+                        const float *ln_b, const float *W_out, const float *b_out, double *logits,
+                        uint8_t *switch_llm)
+{
+    for (int r = 0; r < R; ++r) {
+        size_t src = row_idx ? (size_t)row_idx[r] : (size_t)r;
+        oracle_router_row(hidden + src * (size_t)d, d, h, ff, n_blocks, W_in, b_in, W1, b1, W2, b2, ln_g, ln_b,
+                          W_out, b_out, logits + 2 * (size_t)r);
+        switch_llm[r] = logits[2 * r + 1] > logits[2 * r] ? 1 : 0;
+    }
+}

@@ -35,7 +35,7 @@ import numpy as np
 __all__ = [
     "Workload", "WORKLOADS", "f32_to_bf16_bits", "bf16_bits_to_f32",
     "bf16_bits_to_f64", "make_w_head", "make_hidden", "make_spans",
-    "make_kv_state", "random_mask",
+    "make_kv_state", "random_mask", "make_router_weights",
 ]
 
 
@@ -193,3 +193,16 @@ def random_mask(B: int, p: float, seed: int) -> np.ndarray:
     """Random routing: each sequence is routed with a fixed probability p; uint8 [B]."""
     rng = _rng(seed, 0x4D, int(round(p * 1000)), B)
     return (rng.uniform(size=B) < p).astype(np.uint8)
+
+
+def make_router_weights(d: int, h: int = 32, ff: int = 64, n_blocks: int = 6, seed: int = 1) -> dict:
+    """Random float32 weights for a router network of the shape the paper sketches (an input projection
+    d -> h, n_blocks feed-forward blocks h -> ff -> h, a normalisation and a two-way head); the scales
+    keep activations O(1).  Only random draws: no arithmetic of the network lives here."""
+    rng = _rng(seed, 0x52)
+    n = lambda *shape, s=1.0: (rng.standard_normal(shape) * s).astype(np.float32)
+    return {"W_in": n(h, d, s=1.0 / math.sqrt(d)), "b_in": n(h, s=0.1),
+            "W1": n(n_blocks, ff, h, s=1.0 / math.sqrt(h)), "b1": n(n_blocks, ff, s=0.1),
+            "W2": n(n_blocks, h, ff, s=0.5 / math.sqrt(ff)), "b2": n(n_blocks, h, s=0.1),
+            "ln_g": (1.0 + 0.1 * rng.standard_normal(h)).astype(np.float32), "ln_b": n(h, s=0.1),
+            "W_out": n(2, h, s=1.0 / math.sqrt(h)), "b_out": n(2, s=0.1)}
