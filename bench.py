@@ -43,6 +43,9 @@ BENCH_WORKLOADS = {
     # plan(SLM), plan(LLM), SLM head on the sequences decoding on the SLM, LLM head on the others,
     # commit(SLM), commit(LLM)
     "alg1_b64": ("c4_slm_b64", "c4_llm_b64"),
+    # R-Stitch+ step: SLM head on 64 sequences, the router on the rows the entropy rule routed, compaction
+    # of the router's refined mask
+    "c4_router": ("c4_slm_b64",),
 }
 
 
@@ -288,6 +291,16 @@ def main() -> int:
         # fitted coefficients printed in the paper's latency-regression appendix (SLM-1.5B, LLM-7B), ms
         lat_models = [rs.LatencyModel(0.000021, 0.000231, -0.121046, 27.090929),
                       rs.LatencyModel(0.000027, 0.000031, -0.045256, 27.040801)]
+    with_router = args.workload == "c4_router"
+    router = None
+    if with_router:
+        d0 = gen.WORKLOADS[names[0]].d
+        rw = gen.make_router_weights(d0, 32, 64, 6, seed=77)      # 0.07 M parameters at d = 1536
+        router = rs.Router({k: torch.from_numpy(v).to(dev) for k, v in rw.items()})
+        r_logits = torch.zeros((64, 2), dtype=torch.float32, device=dev)
+        r_switch = torch.zeros(64, dtype=torch.uint8, device=dev)
+        r_idx = torch.zeros(64, dtype=torch.int32, device=dev)
+        r_cnt = torch.zeros(1, dtype=torch.int32, device=dev)
     handles, prepared = [], [[] for _ in range(n_rot)]
     prev_out = [None] * n_rot
     algo_bytes = 0
@@ -331,12 +344,17 @@ def main() -> int:
         if alg1:
             for m in (0, 1):
                 state.commit(m, calls[m].out.tok, calls[m].out.mask, -1, spans=False, stream=stream)
+        if with_router:
+            o = calls[0].out
+            router.forward(calls[0]._keep[1], 64, row_idx=o.llm_idx, n_rows_dev=o.llm_count, logits=r_logits,
+                           switch=r_switch, refine_mask=o.mask, stream=stream)
+            rs.compact(o.mask, r_idx, r_cnt, stream=stream)
 
     for i in range(Wm):
         step(i)
     torch.cuda.synchronize()
     warm_launches = sum(rs.last_status(hd)["launches"] for hd in handles)     # also clears the counters
-    launches_per_step = warm_launches / float(Wm) + (4 if alg1 else 0)
+    launches_per_step = warm_launches / float(Wm) + (4 if alg1 else 0) + (2 if with_router else 0)
 
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if dist is not None:
@@ -382,7 +400,7 @@ def main() -> int:
         dist.barrier()
     ms = ev0.elapsed_time(ev1)
     stats = [rs.last_status(hd) for hd in handles]
-    launches = sum(st["launches"] for st in stats) + (4 * K if alg1 else 0)
+    launches = sum(st["launches"] for st in stats) + (4 * K if alg1 else 0) + (2 * K if with_router else 0)
     if graph is not None:
         launches = int(round(K * launches_per_step))      # replayed kernels are not counted by the handles
     if any(st["timeouts"] or st["nan_rows"] for st in stats):

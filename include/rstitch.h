@@ -259,6 +259,36 @@ int rstitch_alg1_commit(const rstitch_alg1_state_t *s, int B, int model, const i
                         const int32_t *run_count, const int32_t *row_off, const int32_t *tok,
                         const uint8_t *route_mask, int32_t eos_id, void *cuda_stream);
 
+/* ---- R-Stitch+ router ---------------------------------------------------------------------------- */
+
+/*
+ * Weights of the lightweight router (the appendix "Architecture and Overhead of Router": 6 FFN blocks
+ * with GELU and residual connections, a normalisation, a two-head linear layer, on the hidden state;
+ * widths are not given in the paper and are parameters here).  DEVICE pointers to float32, row-major:
+ *   W_in [h, d], b_in [h]            x0 = W_in s + b_in
+ *   W1 [n_blocks, ff, h], b1 [n_blocks, ff], W2 [n_blocks, h, ff], b2 [n_blocks, h]
+ *                                    x <- x + W2 GELU(W1 x + b1) + b2   (exact erf GELU)
+ *   ln_g [h], ln_b [h]               y = LayerNorm(x) ln_g + ln_b       (eps 1e-5)
+ *   W_out [2, h], b_out [2]          logits = W_out y + b_out           (index 0 = SLM, 1 = LLM)
+ * Limits: h <= 256, ff <= 1024, d <= 16384.
+ */
+typedef struct rstitch_router_s {
+    int32_t d, h, ff, n_blocks;
+    const float *W_in, *b_in, *W1, *b1, *W2, *b2, *ln_g, *ln_b, *W_out, *b_out;
+} rstitch_router_t;
+
+/*
+ * Algorithm 1, R-Stitch+ branch: for the rows whose entropy exceeded tau, switch = (argmax_a pi(a | s_t)
+ * == LLM).  Row r reads hidden[row_idx[r]] (bf16 [n_src, d]; row_idx optional) -- typically row_idx =
+ * llm_idx and n_rows_dev = llm_count of the SLM head's call, both on the device.
+ *   logits_out  float32 [R, 2];  switch_out optional uint8 [R] (1 = hand the step to the LLM; a tie keeps
+ *   the SLM);  refine_mask optional uint8 [n_src] (needs row_idx): refine_mask[row_idx[r]] = switch, which
+ *   turns the entropy rule's route_mask into the router's; compact it again with rstitch_compact.
+ */
+int rstitch_router_forward(const rstitch_router_t *w, const void *hidden, int n_src, const int32_t *row_idx,
+                           const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out,
+                           uint8_t *refine_mask, void *cuda_stream);
+
 /* Handle: owns the scratch memory and the device status word for problems up to the given maxima on
  * the current device.  rstitch_destroy(NULL) is a no-op. */
 int rstitch_create(rstitch_handle_t *out, int maxR, int max_d, int maxV);

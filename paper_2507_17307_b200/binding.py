@@ -23,7 +23,7 @@ EXPORTS = [
     "rstitch_route", "rstitch_route_ex", "rstitch_route_host", "rstitch_create", "rstitch_destroy",
     "rstitch_workspace_bytes", "rstitch_compact", "rstitch_last_status", "rstitch_status_string",
     "rstitch_path_name", "rstitch_route_static", "rstitch_route_ex_host",
-    "rstitch_alg1_init", "rstitch_alg1_plan", "rstitch_alg1_commit",
+    "rstitch_alg1_init", "rstitch_alg1_plan", "rstitch_alg1_commit", "rstitch_router_forward",
 ]
 
 
@@ -61,6 +61,14 @@ class DevStat(C.Structure):
 class LatencyModel(C.Structure):
     """rstitch_latency_model_t: Eq. 5 coefficients (a, b, c, d), milliseconds."""
     _fields_ = [("a", C.c_double), ("b", C.c_double), ("c", C.c_double), ("d", C.c_double)]
+
+
+ROUTER_KEYS = ("W_in", "b_in", "W1", "b1", "W2", "b2", "ln_g", "ln_b", "W_out", "b_out")
+
+
+class _Router(C.Structure):
+    _fields_ = [("d", C.c_int32), ("h", C.c_int32), ("ff", C.c_int32), ("n_blocks", C.c_int32)] + \
+               [(k, C.c_void_p) for k in ROUTER_KEYS]
 
 
 class _Alg1State(C.Structure):
@@ -107,6 +115,8 @@ def lib():
         L.rstitch_path_name.restype = C.c_char_p
         L.rstitch_route_static.argtypes = [vp, vp, i, i, i, f, vp, vp, vp, vp, vp, vp]
         L.rstitch_route_static.restype = i
+        L.rstitch_router_forward.argtypes = [C.POINTER(_Router), vp, i, vp, vp, i, vp, vp, vp, vp]
+        L.rstitch_router_forward.restype = i
         L.rstitch_alg1_init.argtypes = [C.POINTER(_Alg1State), i, vp, vp]
         L.rstitch_alg1_init.restype = i
         L.rstitch_alg1_plan.argtypes = [C.POINTER(_Alg1State), i, i, i, C.POINTER(LatencyModel), vp, vp, vp, vp, vp, vp]
@@ -431,3 +441,34 @@ class Alg1State:
                                        _ptr(tok), _ptr(mask), int(eos_id), _stream_ptr(stream))
         if st != 0:
             raise RstitchError(st, "rstitch_alg1_commit")
+
+
+class Router:
+    """rstitch_router_t over device tensors (float32): the R-Stitch+ router's weights."""
+
+    def __init__(self, weights: dict):
+        self.w = weights
+        h, d = weights["W_in"].shape
+        L, ff, _ = weights["W1"].shape
+        c = _Router()
+        c.d, c.h, c.ff, c.n_blocks = int(d), int(h), int(ff), int(L)
+        for k in ROUTER_KEYS:
+            setattr(c, k, _ptr(weights[k]))
+        self._c = c
+
+    def forward(self, hidden, R: int, row_idx=None, n_rows_dev=None, logits=None, switch=None, refine_mask=None,
+                stream=None, check: bool = True):
+        """rstitch_router_forward; returns (logits float32 [R, 2], switch uint8 [R])."""
+        import torch
+        if logits is None:
+            logits = torch.zeros((max(R, 1), 2), dtype=torch.float32, device=hidden.device)
+        if switch is None:
+            switch = torch.full((max(R, 1),), 255, dtype=torch.uint8, device=hidden.device)
+        st = lib().rstitch_router_forward(C.byref(self._c), _ptr(hidden), int(hidden.shape[0]), _ptr(row_idx),
+                                          _ptr(n_rows_dev), int(R), _ptr(logits), _ptr(switch), _ptr(refine_mask),
+                                          _stream_ptr(stream))
+        if not check:
+            return st
+        if st != 0:
+            raise RstitchError(st, "rstitch_router_forward")
+        return logits, switch

@@ -1,0 +1,92 @@
+"""GPU parity of the R-Stitch+ router forward against the oracle, alone and chained after the routing
+decision (entropy rule -> router on the routed rows -> refined mask -> compaction)."""
+import numpy as np
+import pytest
+
+import rstitch_inputs as gen
+from parity_util import to_dev_bf16, to_dev_i32
+
+pytestmark = pytest.mark.gpu
+LOGIT_TOL = 2e-3
+
+
+@pytest.fixture(scope="module")
+def rs():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2507_17307_b200 import build
+    build.build_library()
+    import paper_2507_17307_b200 as rs
+    return rs
+
+
+def dev_weights(w):
+    import torch
+    return {k: torch.from_numpy(v).cuda() for k, v in w.items()}
+
+
+@pytest.mark.parametrize("R,d,h,ff,L", [(1, 64, 8, 16, 1), (7, 256, 32, 64, 6), (64, 1536, 32, 64, 6),
+                                         (33, 3584, 40, 80, 6), (5, 512, 256, 1024, 2), (3, 128, 16, 32, 0)])
+def test_router_logits_and_switch(rs, oracle, R, d, h, ff, L):
+    import torch
+    w = gen.make_router_weights(d, h, ff, max(L, 1), seed=R + d)
+    if L == 0:
+        w = {k: (v[:0] if k in ("W1", "b1", "W2", "b2") else v) for k, v in w.items()}
+        w["W1"] = np.zeros((0, ff, h), np.float32); w["W2"] = np.zeros((0, h, ff), np.float32)
+        w["b1"] = np.zeros((0, ff), np.float32); w["b2"] = np.zeros((0, h), np.float32)
+    rng = np.random.default_rng(R * 31 + d)
+    hid = gen.f32_to_bf16_bits((rng.standard_normal((R + 3, d)) * 2.0).astype(np.float32))
+    idx = rng.integers(0, R + 3, size=R).astype(np.int32)
+    router = rs.Router(dev_weights(w))
+    for row_idx in (None, idx):
+        ref_logits, ref_sw = oracle.router_rows(hid, w, row_idx=row_idx) if row_idx is not None else \
+            oracle.router_rows(hid[:R], w)
+        logits, sw = router.forward(to_dev_bf16(hid), R, row_idx=None if row_idx is None else to_dev_i32(row_idx))
+        torch.cuda.synchronize()
+        got = logits.cpu().numpy()[:R]
+        assert np.abs(got - ref_logits).max() <= LOGIT_TOL
+        clear = np.abs(ref_logits[:, 1] - ref_logits[:, 0]) > 2 * LOGIT_TOL
+        assert np.array_equal(sw.cpu().numpy()[:R][clear], ref_sw[clear])
+
+
+def test_router_after_the_entropy_rule(rs, oracle):
+    import torch
+    ws = gen.scaled(gen.WORKLOADS["c4_slm_b64"], V=3000, d=512, B=64)
+    w_bits = gen.make_w_head(ws)
+    hid, _ = gen.make_hidden(ws, w_bits, 1)
+    rw = gen.make_router_weights(512, 32, 64, 6, seed=5)
+    handle = rs.Handle(64, 512, 3000)
+    hid_dev = to_dev_bf16(hid)
+    out = rs.route_ex(handle, hid_dev, to_dev_bf16(w_bits), ws.tau_nats)
+    router = rs.Router(dev_weights(rw))
+    mask = out.mask.clone()
+    logits, sw = router.forward(hid_dev, 64, row_idx=out.llm_idx, n_rows_dev=out.llm_count, refine_mask=mask)
+    idx2, cnt2 = rs.compact(mask)
+    torch.cuda.synchronize()
+    ref = oracle.route(hid, w_bits, ws.tau_nats)
+    assert (np.abs(ref["ent"] - ws.tau_nats) > 2e-3).all(), "pick another step: a row sits in the tolerance band"
+    cnt = int(out.llm_count.item())
+    assert cnt == ref["llm_count"] and 0 < cnt < 64
+    r_logits, r_sw = oracle.router_rows(hid, rw, row_idx=ref["llm_idx"])
+    assert np.abs(logits.cpu().numpy()[:cnt] - r_logits).max() <= LOGIT_TOL
+    assert (np.abs(r_logits[:, 1] - r_logits[:, 0]) > 2 * LOGIT_TOL).all()
+    want_mask = np.zeros(64, np.uint8)
+    want_mask[ref["llm_idx"]] = r_sw                      # routed only where the router says LLM
+    assert np.array_equal(mask.cpu().numpy(), want_mask)
+    assert (sw.cpu().numpy()[cnt:] == 255).all()          # entries past the live count are untouched
+    want_idx = np.flatnonzero(want_mask)
+    assert int(cnt2.item()) == want_idx.size and np.array_equal(idx2.cpu().numpy()[:want_idx.size], want_idx)
+    assert 0 < want_idx.size < cnt                        # the router kept some steps on the SLM
+    handle.destroy()
+
+
+def test_router_argument_errors(rs):
+    import torch
+    w = dev_weights(gen.make_router_weights(64, 8, 16, 1, seed=1))
+    r = rs.Router(w)
+    hid = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
+    mask = torch.zeros(4, dtype=torch.uint8, device="cuda")
+    assert r.forward(hid, 4, refine_mask=mask, check=False) == -1            # refine needs row_idx
+    big = rs.Router(dev_weights(gen.make_router_weights(64, 300, 16, 1, seed=1)))
+    assert big.forward(hid, 4, check=False) == -3
+    assert r.forward(hid, 0)[0] is not None                                  # empty batch is fine
