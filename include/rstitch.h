@@ -270,7 +270,7 @@ int rstitch_alg1_commit(const rstitch_alg1_state_t *s, int B, int model, const i
  *                                    x <- x + W2 GELU(W1 x + b1) + b2   (exact erf GELU)
  *   ln_g [h], ln_b [h]               y = LayerNorm(x) ln_g + ln_b       (eps 1e-5)
  *   W_out [2, h], b_out [2]          logits = W_out y + b_out           (index 0 = SLM, 1 = LLM)
- * Limits: h <= 256, ff <= 1024, d <= 16384.
+ * Limits: h <= 256, ff <= 1024, d <= 16384 and a multiple of 4, W_in 16-byte aligned.
  */
 typedef struct rstitch_router_s {
     int32_t d, h, ff, n_blocks;

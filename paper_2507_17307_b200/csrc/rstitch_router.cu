@@ -13,8 +13,29 @@
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 constexpr int kMaxH = 256, kMaxFF = 1024;
+
+__device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                 ::"r"((unsigned)__cvta_generic_to_shared(dst_smem)), "l"(src) : "memory");
+}
+
+__device__ __forceinline__ void cp_async4(float *dst_smem, const float *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
+                 ::"r"((unsigned)__cvta_generic_to_shared(dst_smem)), "l"(src) : "memory");
+}
+
+// All threads of the block: n floats, global -> shared, asynchronously.
+__device__ __forceinline__ const float *stage_small(float *&cursor, const float *src, int n)
+{
+    float *dst = cursor;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) cp_async4(dst + i, src + i);
+    cursor += (n + 3) & ~3;
+    return dst;
+}
 
 __device__ __forceinline__ float warp_sum(float v)
 {
@@ -23,11 +44,12 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 1)
 router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const int32_t *row_idx,
-              const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out, uint8_t *refine_mask)
+              const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out, uint8_t *refine_mask,
+              int stage_weights)
 {
-    extern __shared__ float sm[];                 // [d] hidden row | [h] x | [ff] t
+    extern __shared__ float sm[];                 // [d] hidden row | [h] x | [ff] t | [ff h] W1 | [h ff] W2 of a block
     float *s = sm, *x = sm + w.d, *t = x + w.h;
     int R_live = R;
     if (n_rows_dev) { int n = *n_rows_dev; R_live = n < 0 ? 0 : (n < R ? n : R); }
@@ -37,31 +59,119 @@ router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const
     if (src < 0 || src >= n_src) src = 0;
     const unsigned short *hrow = hidden + (size_t)src * w.d;
     for (int k = threadIdx.x; k < w.d; k += kThreads) s[k] = __uint_as_float((unsigned)hrow[k] << 16);
+    float *blk = t + w.ff;                        // staged block weights
+    const float *p_b_in = w.b_in, *p_b1 = w.b1, *p_b2 = w.b2, *p_ln_g = w.ln_g, *p_ln_b = w.ln_b,
+                *p_W_out = w.W_out, *p_b_out = w.b_out;
+    const int per_block = 2 * w.ff * w.h;
+    if (stage_weights == 2) {
+        // every block's matrices at once with asynchronous 16-byte copies (no registers, no waiting
+        // between them): one trip to L2 that overlaps the projection below
+        const int n4 = (w.ff * w.h) >> 2;
+        for (int l = 0; l < w.n_blocks; ++l) {
+            const float *w1 = w.W1 + (size_t)l * w.ff * w.h, *w2 = w.W2 + (size_t)l * w.h * w.ff;
+            float *dst = blk + (size_t)l * per_block;
+            for (int i = threadIdx.x; i < n4; i += kThreads) {
+                cp_async16(dst + 4 * i, w1 + 4 * i);
+                cp_async16(dst + w.ff * w.h + 4 * i, w2 + 4 * i);
+            }
+        }
+        // and every small vector: a scalar read from global memory inside the layer loops costs a full
+        // trip to L2 each time
+        float *cursor = blk + (size_t)w.n_blocks * per_block;
+        p_b_in = stage_small(cursor, w.b_in, w.h);
+        p_b1 = stage_small(cursor, w.b1, w.n_blocks * w.ff);
+        p_b2 = stage_small(cursor, w.b2, w.n_blocks * w.h);
+        p_ln_g = stage_small(cursor, w.ln_g, w.h);
+        p_ln_b = stage_small(cursor, w.ln_b, w.h);
+        p_W_out = stage_small(cursor, w.W_out, 2 * w.h);
+        p_b_out = stage_small(cursor, w.b_out, 2);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = kThreads / 32;
-    for (int i = warp; i < w.h; i += nwarps) {                       // x0 = W_in s + b_in
-        const float *wr = w.W_in + (size_t)i * w.d;
-        float acc = 0.f;
-        for (int k = lane; k < w.d; k += 32) acc = fmaf(wr[k], s[k], acc);
-        acc = warp_sum(acc);
-        if (lane == 0) x[i] = acc + w.b_in[i];
+    // x0 = W_in s + b_in: sixteen warps, two outputs each at a time, sixteen 16-byte loads in flight
+    // per lane (the projection is latency-bound: a block reads all of W_in from L2 by itself)
+    const int d4 = w.d >> 2;
+    const float4 *s4 = reinterpret_cast<const float4 *>(s);
+    for (int i0 = warp * 2; i0 < w.h; i0 += nwarps * 2) {
+        float acc[2] = {0.f, 0.f};
+        const float4 *wr[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) wr[q] = reinterpret_cast<const float4 *>(w.W_in + (size_t)min(i0 + q, w.h - 1) * w.d);
+#pragma unroll 8
+        for (int k = lane; k < d4; k += 32) {
+            const float4 sv = s4[k];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const float4 wv = __ldg(wr[q] + k);
+                acc[q] = fmaf(wv.x, sv.x, fmaf(wv.y, sv.y, fmaf(wv.z, sv.z, fmaf(wv.w, sv.w, acc[q]))));
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const float v = warp_sum(acc[q]);
+            if (lane == 0 && i0 + q < w.h) x[i0 + q] = v;            // the bias joins after the staging wait
+        }
     }
+    __syncthreads();
+    if (stage_weights == 2) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+    }
+    if (threadIdx.x < w.h) x[threadIdx.x] += p_b_in[threadIdx.x];
     __syncthreads();
     for (int l = 0; l < w.n_blocks; ++l) {                          // residual FFN blocks
         const float *w1 = w.W1 + (size_t)l * w.ff * w.h, *w2 = w.W2 + (size_t)l * w.h * w.ff;
-        for (int j = threadIdx.x; j < w.ff; j += kThreads) {
-            float acc = w.b1[(size_t)l * w.ff + j];
-            for (int i = 0; i < w.h; ++i) acc = fmaf(w1[(size_t)j * w.h + i], x[i], acc);
-            t[j] = 0.5f * acc * (1.0f + erff(acc * 0.70710678118654752f));     // exact GELU
+        if (stage_weights == 2) {
+            w1 = blk + (size_t)l * per_block;
+            w2 = w1 + w.ff * w.h;
+        } else if (stage_weights == 1) {
+            // both matrices of the block into shared memory with coalesced, independent loads: one trip
+            // to L2 per block instead of a dependent chain of loads inside the small dot products
+            float *s1 = blk, *s2 = s1 + w.ff * w.h;
+#pragma unroll 8
+            for (int i = threadIdx.x; i < w.ff * w.h; i += kThreads) { s1[i] = __ldg(w1 + i); s2[i] = __ldg(w2 + i); }
+            __syncthreads();
+            w1 = s1; w2 = s2;
+        }
+        // a warp takes four outputs at a time, lanes over the inner index: consecutive shared-memory
+        // words (no bank conflicts), four independent dot products and butterflies in flight (a single
+        // chain of dependent shuffles per output made each block cost ~8000 cycles), and lanes 0-3 apply
+        // the activation to one output each
+        for (int j0 = warp * 4; j0 < w.ff; j0 += nwarps * 4) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int i = lane; i < w.h; i += 32) {
+                const float xi = x[i];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[q] = fmaf(w1[(size_t)min(j0 + q, w.ff - 1) * w.h + i], xi, acc[q]);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], o);
+            }
+            const float mine = lane == 0 ? acc[0] : (lane == 1 ? acc[1] : (lane == 2 ? acc[2] : acc[3]));
+            if (lane < 4 && j0 + lane < w.ff) {
+                const float a = mine + p_b1[(size_t)l * w.ff + j0 + lane];
+                t[j0 + lane] = 0.5f * a * (1.0f + erff(a * 0.70710678118654752f));      // exact GELU
+            }
         }
         __syncthreads();
-        float add = 0.f;
-        if (threadIdx.x < w.h) {
-            add = w.b2[(size_t)l * w.h + threadIdx.x];
-            for (int j = 0; j < w.ff; ++j) add = fmaf(w2[(size_t)threadIdx.x * w.ff + j], t[j], add);
+        for (int i0 = warp * 4; i0 < w.h; i0 += nwarps * 4) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int j = lane; j < w.ff; j += 32) {
+                const float tj = t[j];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[q] = fmaf(w2[(size_t)min(i0 + q, w.h - 1) * w.ff + j], tj, acc[q]);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], o);
+            }
+            const float mine = lane == 0 ? acc[0] : (lane == 1 ? acc[1] : (lane == 2 ? acc[2] : acc[3]));
+            if (lane < 4 && i0 + lane < w.h) x[i0 + lane] += mine + p_b2[(size_t)l * w.h + i0 + lane];   // residual
         }
-        __syncthreads();
-        if (threadIdx.x < w.h) x[threadIdx.x] += add;
         __syncthreads();
     }
     if (warp == 0) {                                                // LayerNorm and the two-way head
@@ -73,12 +183,12 @@ router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const
         const float inv = rsqrtf(warp_sum(sq) / (float)w.h + 1e-5f);
         float a0 = 0.f, a1 = 0.f;
         for (int i = lane; i < w.h; i += 32) {
-            const float y = (x[i] - mean) * inv * w.ln_g[i] + w.ln_b[i];
-            a0 = fmaf(w.W_out[i], y, a0);
-            a1 = fmaf(w.W_out[w.h + i], y, a1);
+            const float y = (x[i] - mean) * inv * p_ln_g[i] + p_ln_b[i];
+            a0 = fmaf(p_W_out[i], y, a0);
+            a1 = fmaf(p_W_out[w.h + i], y, a1);
         }
-        a0 = warp_sum(a0) + w.b_out[0];
-        a1 = warp_sum(a1) + w.b_out[1];
+        a0 = warp_sum(a0) + p_b_out[0];
+        a1 = warp_sum(a1) + p_b_out[1];
         if (lane == 0) {
             const uint8_t sw = a1 > a0 ? 1 : 0;                     // a tie keeps the SLM
             logits_out[2 * r] = a0;
@@ -104,15 +214,33 @@ extern "C" int rstitch_router_forward(const rstitch_router_t *w, const void *hid
     if (R > 0 && !hidden) return RSTITCH_ERR_INVALID_ARG;
     if (refine_mask && !row_idx) return RSTITCH_ERR_INVALID_ARG;
     if (R == 0) return RSTITCH_OK;
-    const size_t smem = (size_t)(w->d + w->h + w->ff) * sizeof(float);
-    if (smem > 48 * 1024) {
+    if (w->d % 4 != 0) return RSTITCH_ERR_UNSUPPORTED_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(w->W_in) & 15u) != 0) return RSTITCH_ERR_BAD_ALIGN;     // read 16 bytes at a time
+    size_t smem = (size_t)(w->d + w->h + w->ff) * sizeof(float);
+    const size_t one = 2 * (size_t)w->h * w->ff * sizeof(float);
+    // 2: all blocks' matrices staged at once; 1: one block at a time; 0: large widths read them from L2
+    int stage_weights = 0;
+    const bool aligned16 = ((reinterpret_cast<uintptr_t>(w->W1) | reinterpret_cast<uintptr_t>(w->W2)) & 15u) == 0 &&
+                           (w->h * w->ff) % 4 == 0 && (w->d + w->h + w->ff) % 4 == 0;
+    const size_t small = (size_t)(w->h * 6 + w->n_blocks * (w->ff + w->h) + 64) * sizeof(float);
+    if (aligned16 && smem + one * (size_t)w->n_blocks + small <= 200 * 1024) {
+        stage_weights = 2;
+        smem += one * (size_t)w->n_blocks + small;
+    }
+    else if (smem + one <= 200 * 1024)                  { stage_weights = 1; smem += one; }
+    static size_t configured[64] = {};       // largest dynamic shared memory asked for so far, per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    if (smem > 48 * 1024 && smem > configured[dev]) {
         if (cudaFuncSetAttribute(router_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
             cudaGetLastError();
             return RSTITCH_ERR_CUDA;
         }
+        configured[dev] = smem;
     }
     router_kernel<<<R, kThreads, smem, (cudaStream_t)cuda_stream>>>(*w, (const unsigned short *)hidden, n_src, row_idx,
-                                                                    n_rows_dev, R, logits_out, switch_out, refine_mask);
+                                                                    n_rows_dev, R, logits_out, switch_out, refine_mask,
+                                                                    stage_weights);
     if (cudaGetLastError() != cudaSuccess) return RSTITCH_ERR_CUDA;
     return RSTITCH_OK;
 }
