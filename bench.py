@@ -225,6 +225,131 @@ def run_reference(args, names) -> dict:
     }
 
 
+def run_vocab_parallel(args, names, rank, local_rank, world) -> int:
+    """The head split by vocabulary rows over the ranks: every rank runs the head kernels on its rows of
+    W_head for ALL rows of the batch, one all-gather moves 20 bytes per row and rank, every rank merges
+    and decides.  Total work is fixed as ranks are added ("strong")."""
+    import torch
+    import paper_2507_17307_b200 as rs
+    from paper_2507_17307_b200 import build as rs_build, sharding
+    if rank == 0:
+        rs_build.build_library()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    rs.lib()
+    dev = torch.device("cuda", local_rank)
+    K = args.steps if args.steps is not None else 4096
+    Wm = max(args.warmup if args.warmup is not None else 64, 3)
+    n_rot = 8
+    head = build_batches(names[:1], n_rot, 0)[0]          # every rank sees the same rows
+    w = head["w"]
+    v_lo, v_hi = sharding.vocab_shard(w.V, rank, world)
+    w_dev = torch.from_numpy(head["w_bits"][v_lo:v_hi].view(np.int16)).to(dev).view(torch.bfloat16)
+    hd = rs.Handle(max(w.B, 64), w.d, w.V)
+    stream = torch.cuda.current_stream()
+    hid_dev = [torch.from_numpy(b["hid"].view(np.int16)).to(dev).view(torch.bfloat16) for b in head["batches"]]
+    hid_pin = [torch.from_numpy(b["hid"].view(np.int16)).view(torch.bfloat16).pin_memory() for b in head["batches"]]
+    mine = torch.zeros((w.B, rs.SHARD_WORDS), dtype=torch.int32, device=dev)
+    gathered = torch.zeros((world, w.B, rs.SHARD_WORDS), dtype=torch.int32, device=dev)
+    outs = [rs.RouteOutputs.allocate(w.B, w.B, dev) for _ in range(n_rot)]
+
+    def step(i, hid=None):
+        j = i % n_rot
+        rs.shard_stats(hd, hid_dev[j] if hid is None else hid, w_dev, v_lo, flags=args.flags, stream=stream,
+                       out=mine if world > 1 else gathered[0])
+        if world > 1:
+            sharding.gather_shard_stats(mine, dist, out=gathered)
+        rs.shard_route(hd, gathered, w.V, w.tau_nats, stream=stream, out=outs[j])
+
+    for i in range(Wm):
+        step(i)
+    torch.cuda.synchronize()
+    rs.last_status(hd)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(visible_gpu_index(local_rank)) as clocks:
+        ev0.record(stream)
+        for i in range(K):
+            step(i)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    ms = ev0.elapsed_time(ev1)
+    st = rs.last_status(hd)
+    if st["timeouts"] or st["nan_rows"]:
+        raise SystemExit("device status after the timed region: %s" % st)
+    launches = st["launches"]
+
+    # end to end: hidden from pinned host memory every step, the decision back in pinned host memory
+    host_out = {k: torch.empty_like(getattr(outs[0], k), device="cpu").pin_memory()
+                for k in ("tok", "ent", "mask", "llm_idx", "llm_count")}
+    stage = torch.empty_like(hid_dev[0])
+
+    def host_step(i):
+        stage.copy_(hid_pin[i % n_rot], non_blocking=True)
+        step(i, stage)
+        for k, t in host_out.items():
+            t.copy_(getattr(outs[i % n_rot], k), non_blocking=True)
+        stream.synchronize()
+
+    Ke = max(1, min(K, 1024))
+    for i in range(3):
+        host_step(i)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for i in range(Ke):
+        host_step(i)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    rs.last_status(hd)
+    ms, _, launches = sharding.reduce_step_stats(ms, 0.0, launches, dist, dev)
+    e2e_s, _, _ = sharding.reduce_step_stats(e2e_s, 0.0, 0, dist, dev)
+    if rank == 0:
+        peaks = measured_peaks()
+        per_step_s = ms / 1e3 / K
+        shard_bytes = (v_hi - v_lo) * w.d * 2               # rank 0's shard, the largest
+        achieved = shard_bytes / per_step_s / 1e9
+        line = {
+            "metric": METRIC, "value": w.B * K / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload + " (vocabulary-parallel)", "B": w.B, "rows_per_step": float(w.B),
+                       "d": w.d, "V": w.V, "tau_nats": w.tau_nats, "heads": list(names[:1]),
+                       "path": [rs.path_name(w.B, w.d, v_hi - v_lo, args.flags)],
+                       "l2": "inputs larger than L2: each step streams the rank's whole W_head shard (%.0f MB); "
+                             "hidden rotates over %d buffers" % (shard_bytes / 1e6, n_rot),
+                       "parallelism": "tp%d (W_head rows sharded, all-gather of %d B per row and rank, every rank "
+                                      "decides)" % (world, 4 * rs.SHARD_WORDS)},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                         "peak_source": "of " + peaks["source"],
+                         "note": "per GPU: the rank's shard bytes over the whole step (head kernel, gather, merge)"},
+            "clocks": clocks.summary(), "gpu_launches": launches,
+            "algorithmic_bytes_per_step": shard_bytes,
+            "e2e": {"value": w.B * Ke / e2e_s, "unit": UNIT, "h2d_bytes_per_step": w.B * w.d * 2,
+                    "d2h_bytes_per_step": sum(t.numel() * t.element_size() for t in host_out.values()),
+                    "steps": Ke, "note": "hidden from pinned host memory, decision back to pinned host memory, "
+                                         "stream synchronised every step; the W_head shard resident"},
+        }
+        print(json.dumps(line), flush=True)
+    hd.destroy()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
 def main() -> int:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -236,6 +361,8 @@ def main() -> int:
     ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="rstitch_args_t.flags (testing)")
     ap.add_argument("--graph", action="store_true",
                     help="capture one rotation of steps into a CUDA graph and time its replays")
+    ap.add_argument("--vocab-parallel", action="store_true",
+                    help="shard W_head by vocabulary rows over the ranks instead of the batch by rows")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -250,6 +377,9 @@ def main() -> int:
         args.warmup = 1 if args.warmup is None else args.warmup
         print(json.dumps(run_reference(args, names)), flush=True)
         return 0
+
+    if args.vocab_parallel:
+        return run_vocab_parallel(args, names, rank, local_rank, world)
 
     import torch
     import paper_2507_17307_b200 as rs

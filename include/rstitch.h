@@ -297,6 +297,43 @@ int rstitch_destroy(rstitch_handle_t h);
 /* Scratch bytes one call of that shape needs (0 for an unsupported shape). */
 size_t rstitch_workspace_bytes(int R, int d, int V);
 
+/* ---- vocabulary-parallel head ------------------------------------------------------------------- */
+
+/*
+ * The LM head split by vocabulary rows across GPUs (tensor-parallel head): GPU g holds W_head rows
+ * [v_base_g, v_base_g + V_g) and every GPU the same hidden rows.  Eq. 1 needs sums over the whole
+ * vocabulary; they come from per-shard statistics, 20 bytes per row, that are gathered and merged:
+ *   1. rstitch_shard_stats on every GPU: the head kernels on the shard, nothing decided;
+ *   2. the caller gathers the shards' outputs into one buffer, shard-major (an all-gather over NCCL;
+ *      this library does no communication);
+ *   3. rstitch_shard_route on any GPU that needs the decision: merge in ascending shard order, then
+ *      entropy, token, Eq. 2, mask, compaction and spans exactly as rstitch_route_ex.
+ * The result equals the single-GPU call on the whole vocabulary up to the rounding order of the merge.
+ *
+ * rstitch_shard_stats reads from *a: hidden, W_head (the shard's rows), R, d, V (= V_g, the shard's row
+ * count), n_src, row_idx, n_rows_dev, flags (RSTITCH_SAMPLE and the path flags), temperature, seed, draw,
+ * workspace; B, tau and every output pointer are ignored.  v_base >= 0 is the global index of the shard's
+ * first row; token indices and the sampling noise use global indices, so the draw does not depend on the
+ * split.  shard_stats: DEVICE, R x RSTITCH_SHARD_WORDS 32-bit words, per row
+ *   float m (largest logit), float s = sum e^(z-m), float u = sum e^(z-m) (z-m), float best score,
+ *   int32 global index of the best entry (INT32_MAX if the shard saw no finite logit).
+ * Rows at or past *n_rows_dev are not written.
+ */
+#define RSTITCH_SHARD_WORDS 5
+#define RSTITCH_MAX_SHARDS  1024
+int rstitch_shard_stats(rstitch_handle_t h, const rstitch_args_t *a, int32_t v_base, void *shard_stats,
+                        void *cuda_stream);
+
+/*
+ * gathered: DEVICE, [n_shards][R][RSTITCH_SHARD_WORDS] words (shard g's shard_stats at word offset
+ * g * R * RSTITCH_SHARD_WORDS), 1 <= n_shards <= RSTITCH_MAX_SHARDS.  Reads from *a: R, B, V (the WHOLE
+ * vocabulary size, which bounds the token index and scales tau with RSTITCH_TAU_NORMALIZED), tau, flags,
+ * row_seq, seq_len, kv_len, n_rows_dev and the output pointers, with the meaning they have in
+ * rstitch_route_ex; hidden, W_head, d, row_idx and workspace are ignored.  One kernel launch.
+ */
+int rstitch_shard_route(rstitch_handle_t h, const rstitch_args_t *a, const void *gathered, int32_t n_shards,
+                        void *cuda_stream);
+
 /* S5 alone: ordered compaction of a uint8 mask [B] into idx [B] and count [1] (warp ballot + prefix
  * sums).  Needs no handle; scratch for very large B is taken from a per-device internal handle. */
 int rstitch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, void *cuda_stream);

@@ -115,6 +115,10 @@ def lib():
         L.rstitch_path_name.restype = C.c_char_p
         L.rstitch_route_static.argtypes = [vp, vp, i, i, i, f, vp, vp, vp, vp, vp, vp]
         L.rstitch_route_static.restype = i
+        L.rstitch_shard_stats.argtypes = [vp, C.POINTER(_Args), C.c_int32, vp, vp]
+        L.rstitch_shard_stats.restype = i
+        L.rstitch_shard_route.argtypes = [vp, C.POINTER(_Args), vp, C.c_int32, vp]
+        L.rstitch_shard_route.restype = i
         L.rstitch_router_forward.argtypes = [C.POINTER(_Router), vp, i, vp, vp, i, vp, vp, vp, vp]
         L.rstitch_router_forward.restype = i
         L.rstitch_alg1_init.argtypes = [C.POINTER(_Alg1State), i, vp, vp]
@@ -248,6 +252,64 @@ def route_ex(handle: Handle, hidden, W_head, tau: float, *, R: Optional[int] = N
         return st
     if st != 0:
         raise RstitchError(st, "rstitch_route_ex")
+    return out
+
+
+SHARD_WORDS = 5
+
+
+def shard_stats(handle: Handle, hidden, W_shard, v_base: int, *, R: Optional[int] = None, row_idx=None,
+                n_rows_dev=None, flags: int = 0, stream=None, out=None, sample=None, check: bool = True):
+    """rstitch_shard_stats: the head on one vocabulary shard (rows [v_base, v_base + len(W_shard)) of the
+    whole W_head).  Returns the int32 tensor [R, SHARD_WORDS] of per-row statistics (float words viewed
+    as int32 so that a gather moves them bit for bit)."""
+    import torch
+    n_src, d = int(hidden.shape[0]), int(hidden.shape[1])
+    if R is None:
+        R = int(row_idx.shape[0]) if row_idx is not None else n_src
+    if out is None:
+        out = torch.zeros((R, SHARD_WORDS), dtype=torch.int32, device=hidden.device)
+    a = _Args()
+    a.hidden, a.W_head = _ptr(hidden), _ptr(W_shard)
+    a.R, a.B, a.d, a.V, a.n_src = R, R, d, int(W_shard.shape[0]), n_src
+    a.flags = int(flags)
+    a.row_idx, a.n_rows_dev = _ptr(row_idx), _ptr(n_rows_dev)
+    if sample is not None:
+        a.flags |= SAMPLE
+        a.temperature, a.seed, a.draw = float(sample[0]), int(sample[1]), int(sample[2])
+    st = lib().rstitch_shard_stats(handle.ptr, C.byref(a), int(v_base), _ptr(out), _stream_ptr(stream))
+    if not check:
+        return st
+    if st != 0:
+        raise RstitchError(st, "rstitch_shard_stats")
+    return out
+
+
+def shard_route(handle: Handle, gathered, V: int, tau: float, *, R: Optional[int] = None, B: Optional[int] = None,
+                row_seq=None, n_rows_dev=None, seq_len=None, kv_len=None, flags: int = 0, stream=None,
+                out: Optional[RouteOutputs] = None, check: bool = True):
+    """rstitch_shard_route: merge of the gathered shards [n_shards, R, SHARD_WORDS] and the routing tail;
+    V is the size of the whole vocabulary."""
+    n_shards = int(gathered.shape[0])
+    if R is None:
+        R = int(gathered.shape[1])
+    if B is None:
+        B = R
+    if out is None:
+        out = RouteOutputs.allocate(R, B, gathered.device, spans=seq_len is not None)
+    a = _Args()
+    a.R, a.B, a.V = R, B, int(V)
+    a.tau, a.flags = float(tau), int(flags)
+    a.row_seq, a.n_rows_dev = _ptr(row_seq), _ptr(n_rows_dev)
+    a.seq_len, a.kv_len = _ptr(seq_len), _ptr(kv_len)
+    a.tok_out, a.ent_out, a.route_mask = _ptr(out.tok), _ptr(out.ent), _ptr(out.mask)
+    a.llm_idx, a.llm_count = _ptr(out.llm_idx), _ptr(out.llm_count)
+    a.llm_span, a.llm_row_off = _ptr(out.llm_span), _ptr(out.llm_row_off)
+    st = lib().rstitch_shard_route(handle.ptr, C.byref(a), _ptr(gathered), n_shards, _stream_ptr(stream))
+    if not check:
+        return st
+    if st != 0:
+        raise RstitchError(st, "rstitch_shard_route")
     return out
 
 

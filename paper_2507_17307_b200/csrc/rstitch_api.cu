@@ -95,9 +95,54 @@ int default_handle(rstitch_handle_s **out, int R, int d, int V)
     return RSTITCH_OK;
 }
 
-int validate(const rstitch_handle_s *h, const rstitch_args_t *a)
+enum ValidateMode { kWholeCall = 0, kShardStats = 1, kShardRoute = 2 };
+
+// kShardStats checks what the head reads (no routing argument), kShardRoute what the tail reads and writes.
+int validate(const rstitch_handle_s *h, const rstitch_args_t *a, ValidateMode mode = kWholeCall)
 {
     if (!h || !a) return RSTITCH_ERR_INVALID_ARG;
+    if (mode == kShardStats) {
+        int st = shape_status(a->R, a->d, a->V);
+        if (st != RSTITCH_OK) return st;
+        if (a->n_src < 0) return RSTITCH_ERR_INVALID_ARG;
+        if ((a->flags & RSTITCH_PATH_GEMV) && (a->flags & RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
+        if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA |
+                         RSTITCH_PATH_PAIR))
+            return RSTITCH_ERR_INVALID_ARG;
+        if ((a->flags & RSTITCH_SAMPLE) && !(std::isfinite(a->temperature) && a->temperature > 0.f))
+            return RSTITCH_ERR_INVALID_ARG;
+        if (a->R > 0 && (!a->hidden || !a->W_head)) return RSTITCH_ERR_INVALID_ARG;
+        if (!aligned(a->hidden, 16) || !aligned(a->W_head, 16)) return RSTITCH_ERR_BAD_ALIGN;
+        if (!aligned(a->row_idx, 4) || !aligned(a->n_rows_dev, 4)) return RSTITCH_ERR_BAD_ALIGN;
+        if (a->workspace) {
+            if (!aligned(a->workspace, 256) || a->workspace_bytes < ws_bytes_for(a->R, a->d, a->V))
+                return RSTITCH_ERR_WORKSPACE;
+        } else if (a->R > h->maxR || a->d > h->max_d || a->V > h->maxV) {
+            return RSTITCH_ERR_UNSUPPORTED_SHAPE;
+        }
+        return RSTITCH_OK;
+    }
+    if (mode == kShardRoute) {
+        if (a->R < 0 || a->B < 0 || a->V < 2) return RSTITCH_ERR_INVALID_ARG;
+        if (a->R > kMaxRows) return RSTITCH_ERR_UNSUPPORTED_SHAPE;
+        if (!std::isfinite(a->tau)) return RSTITCH_ERR_INVALID_ARG;
+        if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA |
+                         RSTITCH_PATH_PAIR))
+            return RSTITCH_ERR_INVALID_ARG;
+        if (!a->llm_count) return RSTITCH_ERR_INVALID_ARG;
+        if (a->row_seq == nullptr && a->B != a->R) return RSTITCH_ERR_INVALID_ARG;
+        if (a->row_seq != nullptr && a->n_rows_dev != nullptr) return RSTITCH_ERR_INVALID_ARG;
+        if ((a->seq_len == nullptr) != (a->kv_len == nullptr)) return RSTITCH_ERR_INVALID_ARG;
+        if (a->seq_len && a->B > 0 && (!a->llm_span || !a->llm_row_off)) return RSTITCH_ERR_INVALID_ARG;
+        if (a->R > 0 && (!a->tok_out || !a->ent_out)) return RSTITCH_ERR_INVALID_ARG;
+        if (a->B > 0 && (!a->route_mask || !a->llm_idx)) return RSTITCH_ERR_INVALID_ARG;
+        if (!aligned(a->tok_out, 4) || !aligned(a->ent_out, 4) || !aligned(a->llm_idx, 4) ||
+            !aligned(a->llm_count, 4) || !aligned(a->row_seq, 4) || !aligned(a->n_rows_dev, 4) ||
+            !aligned(a->seq_len, 4) || !aligned(a->kv_len, 4) || !aligned(a->llm_span, 4) ||
+            !aligned(a->llm_row_off, 4))
+            return RSTITCH_ERR_BAD_ALIGN;
+        return RSTITCH_OK;
+    }
     int st = shape_status(a->R, a->d, a->V);
     if (st != RSTITCH_OK) return st;
     if (a->B < 0 || a->n_src < 0) return RSTITCH_ERR_INVALID_ARG;
@@ -136,6 +181,63 @@ bool use_umma(int R, int d, int V, uint32_t flags)
     if (!umma_shape_ok(R, d, V)) return false;       // tiny shapes stay on the streaming kernel
     if (flags & RSTITCH_PATH_UMMA) return true;
     return R > kGemvMaxRows;
+}
+
+// Validated arguments -> kernels.  With shard_stats the head is a vocabulary shard starting at entry
+// v_base: per-row statistics go to shard_stats and no routing output is touched.
+int enqueue_head(rstitch_handle_s *h, const rstitch_args_t *a, cudaStream_t stream, float *shard_stats,
+                        int v_base)
+{
+    if (!shard_stats && (a->R == 0 || a->B == 0)) {
+        // nothing to evaluate or nothing to decide: the compaction of an empty mask
+        if (cudaMemsetAsync(a->llm_count, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
+        if (a->seq_len && a->llm_row_off &&
+            cudaMemsetAsync(a->llm_row_off, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
+        if (a->R == 0) return RSTITCH_OK;
+    }
+
+    HeadArgs ha;
+    ha.hidden = a->hidden; ha.W = a->W_head; ha.R = a->R; ha.d = a->d; ha.V = a->V;
+    ha.n_src = a->n_src > 0 ? a->n_src : a->R;
+    ha.row_idx = a->row_idx; ha.n_rows_dev = a->n_rows_dev;
+    ha.sample = SampleArgs{};
+    if (a->flags & RSTITCH_SAMPLE) {
+        ha.sample.on = 1;
+        ha.sample.inv_t = 1.0f / a->temperature;
+        ha.sample.k0 = (uint32_t)a->seed; ha.sample.k1 = (uint32_t)(a->seed >> 32);
+        ha.sample.d0 = (uint32_t)a->draw; ha.sample.d1 = (uint32_t)(a->draw >> 32);
+        ha.sample.v0 = (uint32_t)v_base;
+    }
+
+    TailArgs ta;
+    ta.R = a->R; ta.B = a->B; ta.V = a->V;
+    ta.tau = (a->flags & RSTITCH_TAU_NORMALIZED) ? a->tau * logf((float)a->V) : a->tau;
+    ta.row_seq = a->row_seq; ta.seq_len = a->seq_len; ta.kv_len = a->kv_len;
+    ta.tok_out = a->tok_out; ta.ent_out = a->ent_out; ta.route_mask = a->route_mask;
+    ta.llm_idx = a->llm_idx; ta.llm_count = a->llm_count;
+    ta.llm_span = a->llm_span; ta.llm_row_off = a->llm_row_off;
+    ta.stat = h->stat;
+    ta.shard_stats = shard_stats; ta.v_base = v_base;
+
+    void *ws = a->workspace ? a->workspace : h->ws;
+    Scratch sc = scratch_carve(ws);
+    if (a->workspace) {
+        // caller scratch: the ticket must start at zero
+        if (cudaMemsetAsync(sc.ticket, 0, sizeof(unsigned), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
+    }
+    cudaError_t e;
+    int launched = 0;
+    if (use_umma(a->R, a->d, a->V, a->flags)) {
+        // the partials region is sized for the shape the scratch was made for
+        size_t part = a->workspace ? ws_partials_bytes(a->R, a->V) : ws_partials_bytes(h->maxR, h->maxV);
+        e = launch_head_umma(ha, ta, sc, (char *)ws + kWsHeader + part, h->sm_count, stream, &launched,
+                             (a->flags & RSTITCH_PATH_PAIR) != 0);
+    } else {
+        e = launch_head_gemv(ha, ta, sc, h->sm_count, stream, &launched);
+    }
+    h->launch_count += (unsigned)launched;
+    if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    return RSTITCH_OK;
 }
 
 }  // namespace
@@ -201,27 +303,37 @@ int rstitch_route_ex(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_str
     if (st != RSTITCH_OK) return st;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     h->last_stream = stream;
+    return enqueue_head(h, a, stream, nullptr, 0);
+}
 
+int rstitch_shard_stats(rstitch_handle_t h, const rstitch_args_t *a, int32_t v_base, void *shard_stats,
+                        void *cuda_stream)
+{
+    int st = validate(h, a, kShardStats);
+    if (st != RSTITCH_OK) return st;
+    if (v_base < 0 || (a->R > 0 && !shard_stats)) return RSTITCH_ERR_INVALID_ARG;
+    if (!aligned(shard_stats, 4)) return RSTITCH_ERR_BAD_ALIGN;
+    if (a->R == 0) return RSTITCH_OK;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    h->last_stream = stream;
+    return enqueue_head(h, a, stream, (float *)shard_stats, v_base);
+}
+
+int rstitch_shard_route(rstitch_handle_t h, const rstitch_args_t *a, const void *gathered, int32_t n_shards,
+                        void *cuda_stream)
+{
+    int st = validate(h, a, kShardRoute);
+    if (st != RSTITCH_OK) return st;
+    if (n_shards < 1 || n_shards > RSTITCH_MAX_SHARDS || (a->R > 0 && !gathered)) return RSTITCH_ERR_INVALID_ARG;
+    if (!aligned(gathered, 4)) return RSTITCH_ERR_BAD_ALIGN;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    h->last_stream = stream;
     if (a->R == 0 || a->B == 0) {
-        // nothing to evaluate or nothing to decide: the compaction of an empty mask
         if (cudaMemsetAsync(a->llm_count, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
         if (a->seq_len && a->llm_row_off &&
             cudaMemsetAsync(a->llm_row_off, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
         if (a->R == 0) return RSTITCH_OK;
     }
-
-    HeadArgs ha;
-    ha.hidden = a->hidden; ha.W = a->W_head; ha.R = a->R; ha.d = a->d; ha.V = a->V;
-    ha.n_src = a->n_src > 0 ? a->n_src : a->R;
-    ha.row_idx = a->row_idx; ha.n_rows_dev = a->n_rows_dev;
-    ha.sample = SampleArgs{};
-    if (a->flags & RSTITCH_SAMPLE) {
-        ha.sample.on = 1;
-        ha.sample.inv_t = 1.0f / a->temperature;
-        ha.sample.k0 = (uint32_t)a->seed; ha.sample.k1 = (uint32_t)(a->seed >> 32);
-        ha.sample.d0 = (uint32_t)a->draw; ha.sample.d1 = (uint32_t)(a->draw >> 32);
-    }
-
     TailArgs ta;
     ta.R = a->R; ta.B = a->B; ta.V = a->V;
     ta.tau = (a->flags & RSTITCH_TAU_NORMALIZED) ? a->tau * logf((float)a->V) : a->tau;
@@ -230,23 +342,11 @@ int rstitch_route_ex(rstitch_handle_t h, const rstitch_args_t *a, void *cuda_str
     ta.llm_idx = a->llm_idx; ta.llm_count = a->llm_count;
     ta.llm_span = a->llm_span; ta.llm_row_off = a->llm_row_off;
     ta.stat = h->stat;
-
-    void *ws = a->workspace ? a->workspace : h->ws;
-    Scratch sc = scratch_carve(ws);
-    if (a->workspace) {
-        // caller scratch: the ticket must start at zero
-        if (cudaMemsetAsync(sc.ticket, 0, sizeof(unsigned), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
-    }
-    cudaError_t e;
+    ta.shard_stats = nullptr; ta.v_base = 0;
+    Scratch sc = scratch_carve(h->ws);
     int launched = 0;
-    if (use_umma(a->R, a->d, a->V, a->flags)) {
-        // the partials region is sized for the shape the scratch was made for
-        size_t part = a->workspace ? ws_partials_bytes(a->R, a->V) : ws_partials_bytes(h->maxR, h->maxV);
-        e = launch_head_umma(ha, ta, sc, (char *)ws + kWsHeader + part, h->sm_count, stream, &launched,
-                             (a->flags & RSTITCH_PATH_PAIR) != 0);
-    } else {
-        e = launch_head_gemv(ha, ta, sc, h->sm_count, stream, &launched);
-    }
+    cudaError_t e = launch_shard_merge((const float *)gathered, n_shards, a->n_rows_dev, ta, sc.ticket, stream,
+                                       &launched);
     h->launch_count += (unsigned)launched;
     if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
     return RSTITCH_OK;

@@ -44,6 +44,10 @@ size_t      umma_gather_bytes(int R, int d);
 cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
                              int sm_count, cudaStream_t stream, int *launched, bool use_pair);
 
+// Merge of the gathered vocabulary shards ([n_shards][R][5] words, shard-major) and the routing tail.
+cudaError_t launch_shard_merge(const float *gathered, int n_shards, const int32_t *n_rows_dev, const TailArgs &t,
+                               unsigned *ticket, cudaStream_t stream, int *launched);
+
 // Upper bound on the partials per row of any kernel for a vocabulary of V rows.
 __host__ __device__ inline size_t max_slices_for(int V)
 {

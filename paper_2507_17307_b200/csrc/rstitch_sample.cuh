@@ -15,6 +15,8 @@ struct SampleArgs {
     float    inv_t;       // 1 / T_s
     uint32_t k0, k1;      // seed
     uint32_t d0, d1;      // draw number
+    uint32_t v0;          // index of this head's first vocabulary entry in the whole vocabulary
+                          // (non-zero for a vocabulary shard: the noise of an entry does not depend on the split)
 };
 
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
@@ -62,6 +64,7 @@ __device__ __forceinline__ float gumbel_from_bits(uint32_t x)
 __device__ __forceinline__ float sample_score(const SampleArgs &sa, float z, uint32_t row, uint32_t v)
 {
     uint32_t o[4];
+    v += sa.v0;
     philox4x32_10(v >> 2, row, sa.d0, sa.d1, sa.k0, sa.k1, o);
     const uint32_t x = (v & 2u) ? ((v & 1u) ? o[3] : o[2]) : ((v & 1u) ? o[1] : o[0]);
     return fmaf(z, sa.inv_t, gumbel_from_bits(x));

@@ -91,6 +91,7 @@ extern "C" int rstitch_route_static(const void *hidden, const void *W_head, int 
     ta.tok_out = tok_out; ta.ent_out = ent_out; ta.route_mask = route_mask;
     ta.llm_idx = llm_idx; ta.llm_count = llm_count; ta.llm_span = nullptr; ta.llm_row_off = nullptr;
     ta.stat = (DevStat *)((char *)base + kStatOffset);
+    ta.shard_stats = nullptr; ta.v_base = 0;
     Scratch sc = scratch_carve(base);
     cudaError_t e = launch_head_gemv(ha, ta, sc, sms, stream);
     if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }

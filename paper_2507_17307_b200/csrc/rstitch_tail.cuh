@@ -63,11 +63,25 @@ struct TailArgs {
     int32_t *llm_idx, *llm_count;
     int32_t *llm_span, *llm_row_off;   // optional
     DevStat *stat;
+    // Vocabulary-shard mode: when shard_stats is set the head covers only entries [v_base, v_base + V) of
+    // the vocabulary; each row's merged statistics go out as five words (m, s, u, best score, global
+    // index of the best entry) and nothing is decided: shard_merge_kernel does that on the gathered shards.
+    float   *shard_stats;        // [R][5] or nullptr
+    int      v_base;
 };
+
+constexpr int kShardWords = 5;
 
 // Writes ent_out / tok_out of one row from its merged statistics.
 __device__ __forceinline__ void tail_emit_row(const Stats &t, int r, const TailArgs &a)
 {
+    if (a.shard_stats) {
+        float *o = a.shard_stats + (size_t)r * kShardWords;
+        const bool found = !(t.bi == INT_MAX || t.bi < 0 || t.bi >= a.V);
+        o[0] = t.m; o[1] = t.s; o[2] = t.u; o[3] = t.bv;
+        o[4] = __int_as_float(found ? t.bi + a.v_base : INT_MAX);
+        return;
+    }
     float H = logf(t.s) - t.u / t.s;
     if (H < 0.f) H = 0.f;                      // rounding below zero; NaN stays NaN
     a.ent_out[r] = H;
@@ -378,6 +392,7 @@ __device__ inline void tail_route_warp(const TailArgs &a)
 
 __device__ inline void tail_route(const TailArgs &a, int *smem)
 {
+    if (a.shard_stats) return;                       // a vocabulary shard decides nothing
     if (a.B <= 32 && a.row_seq == nullptr) { tail_route_warp(a); return; }
     tail_mask(a);
     tail_compact(a.route_mask, a.B, a.seq_len, a.kv_len, a.llm_idx, a.llm_count, a.llm_span,

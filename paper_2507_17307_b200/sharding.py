@@ -2,8 +2,15 @@
 
 The path shards by rows: sequences are independent, so every rank decides its own sequences against
 a replicated LM head and there is no data-path collective.  What crosses ranks is only bookkeeping:
-which sequences a rank owns, the slowest rank's time, and the totals.  Nothing here computes any
-part of the decision; it works on CPU tensors with the gloo backend and on CUDA tensors with NCCL.
+which sequences a rank owns, the slowest rank's time, and the totals.
+
+A head too large for one GPU shards by vocabulary rows instead (tensor-parallel head): every rank runs the
+head kernels on its rows of W_head and leaves five words of softmax statistics per row; one all-gather
+of those (20 bytes per row and rank) is the path's only collective, after which each rank merges and
+decides (binding.shard_stats / binding.shard_route).
+
+Nothing here computes any part of the decision; it works on CPU tensors with the gloo backend and on
+CUDA tensors with NCCL.
 """
 from __future__ import annotations
 
@@ -49,3 +56,41 @@ def gather_counts(count: int, dist=None, device="cpu"):
     out = [torch.zeros_like(mine) for _ in range(dist.get_world_size())]
     dist.all_gather(out, mine)
     return [int(o.item()) for o in out]
+
+
+def vocab_shard(V: int, rank: int, world: int, align: int = 16) -> Tuple[int, int]:
+    """[begin, end) of the W_head rows rank `rank` holds when a vocabulary of V entries is split into
+    `world` contiguous shards.  Boundaries are multiples of `align` rows (whole tensor-core tile units),
+    sizes differ by at most `align`, and the last shard takes the ragged end."""
+    if world < 1 or not (0 <= rank < world) or V < 0 or align < 1:
+        raise ValueError("bad sharding arguments")
+    b, e = rank_rows(-(-V // align), rank, world)
+    return min(b * align, V), min(e * align, V)
+
+
+def empty_shard_stats(R: int, device="cpu"):
+    """Statistics of a shard that holds no vocabulary entry (the empty set of the merge): what a rank
+    contributes when the split leaves it no rows.  The head kernels need at least two rows per shard."""
+    import torch
+    import struct
+    ninf = struct.unpack("<i", struct.pack("<f", float("-inf")))[0]
+    row = torch.tensor([ninf, 0, 0, ninf, 2**31 - 1], dtype=torch.int32, device=device)
+    return row.repeat(R, 1)
+
+
+def gather_shard_stats(stats, dist=None, out=None):
+    """All-gather of the per-row shard statistics ([R, 5] int32, every rank the same R) into
+    [world, R, 5] in rank order = ascending vocabulary order, the order the merge wants."""
+    import torch
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        g = stats.unsqueeze(0)
+        if out is not None:
+            out.copy_(g)
+            return out
+        return g
+    world = dist.get_world_size()
+    if out is None:
+        out = torch.empty((world,) + tuple(stats.shape), dtype=stats.dtype, device=stats.device)
+    # the ranks' blocks concatenated along the first axis: the form every backend accepts
+    dist.all_gather_into_tensor(out.view((world * stats.shape[0],) + tuple(stats.shape[1:])), stats.contiguous())
+    return out
