@@ -133,14 +133,14 @@ def measured_peaks() -> dict:
 # once any of them has changed the counters no longer describe the kernel and the figure reads null.
 NCU_TRAFFIC = {
     "c2_slm_b1":
-    {"bytes": 470720256, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
-     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "9b926ebd1d559dc9a04ae4c80c5207d485f26a73d6e19ed5c004030677832df1", "rstitch_tail.cuh": "213850b579815c8438459e1885c78989dfc75244b76a8d4197f62012dd3a097f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "248e633f5dbc3c719b09cc1f421c09ead4e2f15e7339d91091252fd0c3e72569"}},
+    {"bytes": 471029248, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
+     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "d5767ba87bc635bf71f9069bcd7b408ff46f8339a455a5ff627f7a6bec3cbdb6", "rstitch_tail.cuh": "c7354c820b08678c99a76fe9f95332a64ac1a839c76083648825f9da6ec8ad71", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
     "c4_slm_b64":
-    {"bytes": 471161344, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
-     "sources": {"rstitch_umma.cu": "49c9d68e6d65fcbfe0dd5965a2fe5c9e3b6c4962d5bcbed311c70afbe593b9b5", "rstitch_kernels.cuh": "9b926ebd1d559dc9a04ae4c80c5207d485f26a73d6e19ed5c004030677832df1", "rstitch_tail.cuh": "213850b579815c8438459e1885c78989dfc75244b76a8d4197f62012dd3a097f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "248e633f5dbc3c719b09cc1f421c09ead4e2f15e7339d91091252fd0c3e72569"}},
+    {"bytes": 471211008, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
+     "sources": {"rstitch_umma.cu": "95c15fe676ede5ff8503be2afab0782f79839b0f0a88734d0bec3a0ae4a4bba9", "rstitch_kernels.cuh": "d5767ba87bc635bf71f9069bcd7b408ff46f8339a455a5ff627f7a6bec3cbdb6", "rstitch_tail.cuh": "c7354c820b08678c99a76fe9f95332a64ac1a839c76083648825f9da6ec8ad71", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
     "c5_catchup":
-    {"bytes": 1672081912, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
-     "sources": {"rstitch_umma.cu": "49c9d68e6d65fcbfe0dd5965a2fe5c9e3b6c4962d5bcbed311c70afbe593b9b5", "rstitch_kernels.cuh": "9b926ebd1d559dc9a04ae4c80c5207d485f26a73d6e19ed5c004030677832df1", "rstitch_tail.cuh": "213850b579815c8438459e1885c78989dfc75244b76a8d4197f62012dd3a097f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "248e633f5dbc3c719b09cc1f421c09ead4e2f15e7339d91091252fd0c3e72569"}},
+    {"bytes": 1668683672, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
+     "sources": {"rstitch_umma.cu": "95c15fe676ede5ff8503be2afab0782f79839b0f0a88734d0bec3a0ae4a4bba9", "rstitch_kernels.cuh": "d5767ba87bc635bf71f9069bcd7b408ff46f8339a455a5ff627f7a6bec3cbdb6", "rstitch_tail.cuh": "c7354c820b08678c99a76fe9f95332a64ac1a839c76083648825f9da6ec8ad71", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
 }
 
 
