@@ -455,6 +455,57 @@ __device__ __forceinline__ Item2 item2(int q, int nMG, int nM, int V)
     return it;
 }
 
+// Work of one block of head_umma2_kernel.  Items q = 0 .. total-1 are dealt round-robin: block c takes
+// c, c + grid, ...  The last, partly filled round would leave most blocks idle for a whole item, so when
+// its items split into at most `grid` single-M-tile pieces they are dealt as such, one piece per block
+// (a piece costs ~0.6 of a two-tile item: its own hidden tile plus the whole W tile).
+struct Sched2 {
+    int nM, nMG, grid, cta;
+    int n_items;                 // whole items of this block
+    int piece_q, piece_mt;       // this block's piece of the last round (piece_q < 0: none)
+};
+
+__device__ __forceinline__ int tiles_of_item2(int q, int nMG, int nM)
+{
+    const int mg = q % nMG;
+    return (2 * mg + 1 < nM) ? 2 : 1;
+}
+
+__device__ __forceinline__ Sched2 sched2_make(int nM, int V, int grid, int cta, bool any_rows)
+{
+    Sched2 s;
+    s.nM = nM; s.nMG = (nM + 1) / 2; s.grid = grid; s.cta = cta;
+    s.piece_q = -1; s.piece_mt = 0;
+    const int total = ((V + kTileNMax - 1) / kTileNMax) * s.nMG;
+    const int full = (total / grid) * grid;              // items of the completely filled rounds
+    int pieces = 0;
+    for (int q = full; q < total; ++q) pieces += tiles_of_item2(q, s.nMG, nM);
+    if (!any_rows) { s.n_items = 0; return s; }
+    if (pieces > grid || pieces == 0) {                  // nothing to split, or too many pieces: plain deal
+        s.n_items = cta < total ? (total - cta + grid - 1) / grid : 0;
+        return s;
+    }
+    s.n_items = full / grid;
+    int k = 0;
+    for (int q = full; q < total; ++q) {
+        const int n = tiles_of_item2(q, s.nMG, nM);
+        if (cta >= k && cta < k + n) { s.piece_q = q; s.piece_mt = cta - k; }
+        k += n;
+    }
+    return s;
+}
+
+__device__ __forceinline__ int sched2_count(const Sched2 &s) { return s.n_items + (s.piece_q >= 0 ? 1 : 0); }
+
+__device__ __forceinline__ Item2 sched2_item(const Sched2 &s, int j, int V)
+{
+    if (j < s.n_items) return item2(s.cta + j * s.grid, s.nMG, s.nM, V);
+    Item2 it = item2(s.piece_q, s.nMG, s.nM, V);
+    it.m0 += s.piece_mt;                                 // one M tile of the pair, in the first accumulator
+    it.two = 0;
+    return it;
+}
+
 __global__ void __launch_bounds__(kThreads2, 1)
 head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_constant__ WMaps tm_w,
                   HeadArgs h, TailArgs t, Partials P, int nM, int n_slices)
@@ -470,10 +521,8 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
     const int nK = (h.d + kTileK - 1) / kTileK;
     int R_live = h.R;
     if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
-    const int nMG = (nM + 1) / 2;
-    const int total = ((h.V + kTileNMax - 1) / kTileNMax) * nMG;
-    const int cta = blockIdx.x, grid = gridDim.x;
-    const int n_items = (cta < total && R_live > 0) ? (total - cta + grid - 1) / grid : 0;
+    const Sched2 sch = sched2_make(nM, h.V, (int)gridDim.x, (int)blockIdx.x, R_live > 0);
+    const int n_items = sched2_count(sch);
 
     if (threadIdx.x == 0) {
         s_abort = 0; s_zero = 0;
@@ -504,7 +553,7 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
             int stage = 0, round = 0, issued = 0;
             bool live = true;
             for (int j = 0; live && j < n_items; ++j) {
-                const Item2 it = item2(cta + j * grid, nMG, nM, h.V);
+                const Item2 it = sched2_item(sch, j, h.V);
                 for (int ks = 0; ks < nK; ++ks) {
                     if (!ptx::mbar_wait(ptx::smem_u32(&s_empty[stage]), (uint32_t)((round & 1) ^ 1), &s_abort)) {
                         if (!s_abort) raise_abort(&s_abort, t.stat, 0x211u);
@@ -548,7 +597,7 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
             int stage = 0, round = 0;
             bool live = true;
             for (int j = 0; live && j < n_items; ++j) {
-                const Item2 it = item2(cta + j * grid, nMG, nM, h.V);
+                const Item2 it = sched2_item(sch, j, h.V);
                 if (!ptx::mbar_wait(ptx::smem_u32(&s_acc_empty), (uint32_t)((j & 1) ^ 1), &s_abort)) {
                     if (!s_abort) raise_abort(&s_abort, t.stat, 0x212u);
                     break;
@@ -595,7 +644,7 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
         const int mt = (warp - 2) >> 2;
         const int quarter = warp & 3;
         for (int j = 0; j < n_items; ++j) {
-            const Item2 it = item2(cta + j * grid, nMG, nM, h.V);
+            const Item2 it = sched2_item(sch, j, h.V);
             const int rows_per_quarter = tile_is_small(it.m0 + mt, h.R) ? 16 : 32;     // M = 64: 16 rows per quarter
             const int row0 = (it.m0 + mt) * kTileM + quarter * rows_per_quarter;
             const int row = row0 + lane;
