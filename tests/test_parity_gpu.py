@@ -452,3 +452,19 @@ def test_step_loop_replays_from_a_cuda_graph(rs, handle, oracle):
         n = cnt if i in (4, 5) else a.shape[0]          # the LLM head wrote only the routed rows
         assert torch.equal(a[:n], b[:n]), i
     h2.destroy()
+
+
+@pytest.mark.parametrize("B,d,V,path", [(16384, 64, 512, "umma"), (16384, 64, 300, "gemv"), (3, 16384, 300, "gemv"),
+                                         (5, 16384, 512, "umma"), (200, 16384, 256, "umma")])
+def test_maximum_sizes(rs, oracle, B, d, V, path):
+    # the largest row count and the largest hidden size the library accepts, each beside a small other side
+    flag = rs.PATH_GEMV if path == "gemv" else rs.PATH_UMMA
+    h = rs.Handle(B, d, V)
+    try:
+        w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=d, V=V, seed=9700 + B + d + V, sigma_w=0.5 / math.sqrt(d))
+        check_case(rs, h, oracle, w, [0], flags=flag)
+        assert rs.route_ex(h, to_dev_bf16(np.zeros((B, d), dtype=np.uint16)), to_dev_bf16(gen.make_w_head(w)),
+                           0.3, R=B + 1, check=False) != 0        # one row more than the handle was made for
+    finally:
+        h.destroy()
+    assert rs.workspace_bytes(16385, 64, 512) == 0 and rs.workspace_bytes(4, 16392, 512) == 0
