@@ -32,7 +32,8 @@ constexpr int kProducers = 1;                        // copy-issuing warps.  One
                                                      // microsecond and separate warps issue in parallel (a probe reached
                                                      // 19/us with four), but these kernels need at most ~6/us and measured
                                                      // the same with 1, 2 and 3; the dealing code below stays general
-constexpr int kThreads   = 192 + (kProducers - 1) * 32;   // producer, MMA, 4 epilogue warps, extra producers
+constexpr int kEpiWarps  = 8;
+constexpr int kThreads   = 64 + kEpiWarps * 32;      // head_umma_kernel: producer, MMA, 8 epilogue warps
 constexpr int kMaxStages = 8;
 constexpr int kTileM     = 128;
 constexpr int kTileNMax  = 256;
@@ -43,49 +44,31 @@ constexpr int kRingBytes = 224 * 1024;                     // cut into as many s
 constexpr int kDynSmem   = kRingBytes + 1024;              // + slack to align the ring to 1024 B
 constexpr int kTmemCols  = 512;
 
-struct Item { int v0, N, m; };
+struct Item { int v0, N; };
 
-// The work item a block takes at its j-th iteration; identical in every role of the block.
+// The W tile head_umma_kernel's block takes at its j-th iteration; identical in every role of the block.
+// Each block owns a balanced contiguous vocabulary range in units of 16 rows, cut into n_tiles tiles.
 struct Schedule {
-    int V, nM, grid, cta;
-    // one M tile: balanced contiguous ranges in units of 16 vocabulary rows
     int u_begin, nu, n_tiles;
-    // several M tiles
     int n_items;
 
     // tiles_per_block: the same for every block (from the largest range), so that no block's
     // tile exceeds the tile size the shared-memory stages were laid out for
-    __device__ void init(int V_, int nM_, int grid_, int cta_, int tiles_per_block)
+    __device__ void init(int V, int grid, int cta, int tiles_per_block)
     {
-        V = V_; nM = nM_; grid = grid_; cta = cta_;
-        if (nM == 1) {
-            long long units = (V + 15) / 16;
-            u_begin = (int)(units * cta / grid);
-            int u_end = (int)(units * (cta + 1) / grid);
-            nu = u_end - u_begin;
-            n_tiles = tiles_per_block;
-            n_items = n_tiles;
-        } else {
-            int nVT = (V + kTileNMax - 1) / kTileNMax;
-            int total = nVT * nM;
-            n_items = cta < total ? (total - cta + grid - 1) / grid : 0;
-        }
+        long long units = (V + 15) / 16;
+        u_begin = (int)(units * cta / grid);
+        int u_end = (int)(units * (cta + 1) / grid);
+        nu = u_end - u_begin;
+        n_tiles = tiles_per_block;
+        n_items = n_tiles;
     }
     __device__ Item item(int j) const
     {
         Item it;
-        if (nM == 1) {
-            int a = u_begin + (int)((long long)nu * j / n_tiles);
-            int b = u_begin + (int)((long long)nu * (j + 1) / n_tiles);
-            it.v0 = a * 16; it.N = (b - a) * 16; it.m = 0;
-        } else {
-            int q = cta + j * grid;
-            int vt = q / nM;
-            it.m = q - vt * nM;
-            it.v0 = vt * kTileNMax;
-            int left = V - it.v0;
-            it.N = left >= kTileNMax ? kTileNMax : ((left + 15) / 16) * 16;
-        }
+        int a = u_begin + (int)((long long)nu * j / n_tiles);
+        int b = u_begin + (int)((long long)nu * (j + 1) / n_tiles);
+        it.v0 = a * 16; it.N = (b - a) * 16;
         return it;
     }
 };
@@ -212,7 +195,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
 {
     extern __shared__ unsigned char dyn_smem_raw[];
     __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
-    const int nM = plan.nM, n_slices = plan.n_slices, n_stages = plan.n_stages;
+    const int n_slices = plan.n_slices, n_stages = plan.n_stages;
     __shared__ __align__(8) uint64_t s_acc_full[2], s_acc_empty[2], s_done, s_tailbar;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_tail[66];
@@ -225,7 +208,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
 
     Schedule sch;
-    sch.init(h.V, nM, gridDim.x, blockIdx.x, plan.tiles_per_block);
+    sch.init(h.V, gridDim.x, blockIdx.x, plan.tiles_per_block);
     if (R_live == 0) sch.n_items = 0;          // no live rows (device-side count): nothing to stream
 
     if (threadIdx.x == 0) {
@@ -236,7 +219,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(ptx::smem_u32(&s_acc_full[b]), 1);
-            ptx::mbar_init(ptx::smem_u32(&s_acc_empty[b]), 4);     // one arrival per epilogue warp
+            ptx::mbar_init(ptx::smem_u32(&s_acc_empty[b]), kEpiWarps);   // one arrival per epilogue warp
         }
         ptx::mbar_init(ptx::smem_u32(&s_done), 1);
         ptx::mbar_init(ptx::smem_u32(&s_tailbar), 1);
@@ -253,9 +236,9 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
 
-    if (warp == 0 || warp >= 6) {
-        // ---- producers: the copies of a stage are dealt round-robin to kProducers threads ------
-        const int pid = warp == 0 ? 0 : warp - 5;
+    if (warp == 0) {
+        // ---- producer --------------------------------------------------------------------
+        constexpr int pid = 0;
         if (lane == 0) {
             int stage = 0, round = 0, issued = 0;
             bool live = true;
@@ -274,17 +257,15 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                     // and what the stale rows produce lands in accumulator rows nobody looks at
                     if (pid == 0) {
                         ptx::mbar_arrive_expect_tx(full, (uint32_t)((plan.a_rows + it.N) * kTileK * 2));
-                        ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, it.m * kTileM, full);
+                        ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, 0, full);
                     }
-                    int r = 0, op = 1;
+                    int r = 0;
 #pragma unroll
                     for (int b = 4; b >= 0; --b) {
                         const int rows = 16 << b;
                         if (it.N - r >= rows) {
-                            if (op % kProducers == pid)
-                                ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK, it.v0 + r, full);
+                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK, it.v0 + r, full);
                             r += rows;
-                            ++op;
                         }
                     }
                     ++issued;
@@ -344,44 +325,58 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
         }
         __syncwarp();
     } else {
-        // ---- epilogue --------------------------------------------------------------------
+        // ---- epilogue: warps 2-5 fold the first half of a tile's 32-column chunks, warps 6-9 the rest ----
         const int quarter = warp & 3;                        // the TMEM lanes this warp may read
+        const int half = (warp - 2) >> 2;
         // M = 128: accumulator row i is lane i.  M = 64: row i is lane 32 (i / 16) + i % 16.
         const int rows_per_quarter = plan.m64 ? 16 : 32;
-        const int row_in_tile = quarter * rows_per_quarter + lane;
-        const bool lane_has_row = lane < rows_per_quarter;
+        const int row = quarter * rows_per_quarter + lane;
+        const bool lane_has_row = lane < rows_per_quarter && row < R_live;
+        const bool warp_has_rows = quarter * rows_per_quarter < R_live;
         Stats st = stats_empty();
         for (int j = 0; j < sch.n_items; ++j) {
             const Item it = sch.item(j);
             const int buf = j & 1, use = j >> 1;
-            const int row = it.m * kTileM + row_in_tile;
             if (!ptx::mbar_wait(ptx::smem_u32(&s_acc_full[buf]), (uint32_t)(use & 1), &s_abort)) {
                 if (lane == 0 && !s_abort) raise_abort(&s_abort, t.stat, 0x204u);
                 break;
             }
             ptx::tc_fence_after_sync();
-            const bool warp_has_rows = (it.m * kTileM + quarter * rows_per_quarter) < R_live;
-            if (nM > 1) st = stats_empty();
             if (warp_has_rows) {
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kTileNMax;
-                for (int c0 = 0; c0 < it.N; c0 += 32) {
+                const int n_chunks = (it.N + 31) >> 5;
+                const int c_split = ((n_chunks + 1) >> 1) << 5;
+                const int c_begin = half ? c_split : 0, c_end = half ? it.N : (c_split < it.N ? c_split : it.N);
+                for (int c0 = c_begin; c0 < c_end; c0 += 32) {
                     float z[32];
                     ptx::tmem_ld_32x32(taddr + (uint32_t)c0, z);
                     int n_valid = it.N - c0;
                     if (h.V - (it.v0 + c0) < n_valid) n_valid = h.V - (it.v0 + c0);
                     if (n_valid > 32) n_valid = 32;
-                    if (lane_has_row && row < R_live && n_valid > 0)
+                    if (lane_has_row && n_valid > 0)
                         fold_chunk(st, z, n_valid, it.v0 + c0, h.sample, (uint32_t)row);
                 }
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&s_acc_empty[buf]));
-            if (nM > 1 && lane_has_row && row < R_live)
-                partial_store(P, (size_t)row * n_slices + (size_t)(it.v0 / kTileNMax), st);
         }
-        if (nM == 1 && lane_has_row && row_in_tile < R_live)
-            partial_store(P, (size_t)row_in_tile * n_slices + blockIdx.x, st);
+        // Every accumulator has been drained, so every copy has landed and the ring is idle: the second
+        // half's statistics cross to the first half through it, which writes the block's partial.
+        float *xch = reinterpret_cast<float *>(dyn_smem_raw + (ring - ptx::smem_u32(dyn_smem_raw)));
+        const int slot = (quarter * 32 + lane) * 5;
+        if (half == 1) {
+            xch[slot] = st.m; xch[slot + 1] = st.s; xch[slot + 2] = st.u; xch[slot + 3] = st.bv;
+            xch[slot + 4] = __int_as_float(st.bi);
+        }
+        asm volatile("bar.sync 1, %0;" :: "n"(kEpiWarps * 32) : "memory");
+        if (half == 0 && lane_has_row) {
+            Stats o;
+            o.m = xch[slot]; o.s = xch[slot + 1]; o.u = xch[slot + 2]; o.bv = xch[slot + 3];
+            o.bi = __float_as_int(xch[slot + 4]);
+            stats_merge(st, o);
+            partial_store(P, (size_t)row * n_slices + blockIdx.x, st);
+        }
     }
 
     ptx::tc_fence_before_sync();
@@ -391,9 +386,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
-    if (nM > 1) return;               // several M tiles: a separate kernel merges the partials
-
-    // one M tile: the last block done merges all slices and runs the routing tail
+    // the last block done merges all slices and runs the routing tail
     if (threadIdx.x == 0) {
         unsigned k = atomicAdd(ticket, 1u);
         s_last = (k == (unsigned)(gridDim.x - 1));
