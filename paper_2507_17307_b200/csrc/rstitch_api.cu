@@ -24,12 +24,14 @@ struct rstitch_handle_s {
     // staging of rstitch_route_host
     void    *st = nullptr;  size_t st_bytes = 0;     // staging block of the host-buffer calls
     void    *st_host = nullptr;  size_t st_host_bytes = 0;   // pinned mirror of its output part
+    void    *st_in = nullptr;  size_t st_in_bytes = 0;       // pinned mirror of its input part (small inputs)
     cudaStream_t last_stream = nullptr;
     unsigned launch_count = 0;           // kernels enqueued since the status word was last read
 };
 
 namespace {
 
+constexpr size_t kPackedInputMax = 64 * 1024;   // host-buffer calls: inputs up to this size travel as one copy
 constexpr int kMaxD = 16384;
 constexpr int kMaxRows = 16384;
 
@@ -291,7 +293,7 @@ int rstitch_destroy(rstitch_handle_t h)
 {
     if (!h) return RSTITCH_OK;
     cudaFree(h->ws); cudaFree(h->stat); cudaFree(h->tile_counts); cudaFree(h->st);
-    cudaFreeHost(h->st_host);
+    cudaFreeHost(h->st_host); cudaFreeHost(h->st_in);
     cudaGetLastError();
     delete h;
     return RSTITCH_OK;
@@ -410,13 +412,31 @@ int rstitch_route_ex_host(rstitch_handle_t h, const rstitch_args_t *a, void *cud
         h->st_bytes = off;
     }
     char *base = (char *)h->st;
-    auto h2d = [&](size_t o, const void *src, size_t n) {
-        return n == 0 || cudaMemcpyAsync(base + o, src, n, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-    };
-    bool ok = h2d(o_hid, a->hidden, n_src * a->d * 2);
-    if (ok && a->row_idx) ok = h2d(o_ridx, a->row_idx, R * 4);
-    if (ok && a->row_seq) ok = h2d(o_rseq, a->row_seq, R * 4);
-    if (ok && a->seq_len) ok = h2d(o_slen, a->seq_len, B * 4) && h2d(o_klen, a->kv_len, B * 4);
+    bool ok = true;
+    const size_t in_bytes = o_tok;                  // the inputs lead the staging block
+    if (in_bytes <= kPackedInputMax) {
+        // a decode step's inputs are a few KB: gather them in a pinned mirror of the block's input part
+        // and send them with one copy (each small copy costs microseconds of its own)
+        if (in_bytes > h->st_in_bytes) {
+            if (h->st_in) { cudaFreeHost(h->st_in); h->st_in = nullptr; h->st_in_bytes = 0; }
+            if (cudaMallocHost(&h->st_in, kPackedInputMax) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+            h->st_in_bytes = kPackedInputMax;
+        }
+        char *in = (char *)h->st_in;
+        std::memcpy(in + o_hid, a->hidden, n_src * a->d * 2);
+        if (a->row_idx) std::memcpy(in + o_ridx, a->row_idx, R * 4);
+        if (a->row_seq) std::memcpy(in + o_rseq, a->row_seq, R * 4);
+        if (a->seq_len) { std::memcpy(in + o_slen, a->seq_len, B * 4); std::memcpy(in + o_klen, a->kv_len, B * 4); }
+        ok = cudaMemcpyAsync(base, in, in_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    } else {
+        auto h2d = [&](size_t o, const void *src, size_t n) {
+            return n == 0 || cudaMemcpyAsync(base + o, src, n, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+        };
+        ok = h2d(o_hid, a->hidden, n_src * a->d * 2);
+        if (ok && a->row_idx) ok = h2d(o_ridx, a->row_idx, R * 4);
+        if (ok && a->row_seq) ok = h2d(o_rseq, a->row_seq, R * 4);
+        if (ok && a->seq_len) ok = h2d(o_slen, a->seq_len, B * 4) && h2d(o_klen, a->kv_len, B * 4);
+    }
     if (!ok) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
 
     rstitch_args_t dv = *a;
