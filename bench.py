@@ -39,9 +39,9 @@ BENCH_WORKLOADS = {
     "c2_slm_b1": ("c2_slm_b1",), "c3_llm_b1": ("c3_llm_b1",), "c3_llm_b4": ("c3_llm_b4",),
     "c3_llm_b16": ("c3_llm_b16",), "c4_slm_b64": ("c4_slm_b64",),
     "c4_batched": ("c4_slm_b64", "c4_llm_b64"), "c5_catchup": ("c5_catchup",), "c1_tiny": ("c1_tiny",),
-    # one round of the batched hybrid decode loop (Algorithm 1) for 64 sequences, all on the device:
-    # plan(SLM), plan(LLM), SLM head on the sequences decoding on the SLM, LLM head on the others,
-    # commit(SLM), commit(LLM)
+    # one round of the batched hybrid decode loop (Algorithm 1) for 64 sequences, all on the device, two
+    # launches: the SLM head on the sequences decoding on the SLM, the LLM head on the others, each applying
+    # Algorithm 1's decision block in its own tail, the LLM's call also planning the next round
     "alg1_b64": ("c4_slm_b64", "c4_llm_b64"),
     # R-Stitch+ step: SLM head on 64 sequences, the router on the rows the entropy rule routed, compaction
     # of the router's refined mask
@@ -431,6 +431,7 @@ def main() -> int:
         r_switch = torch.zeros(64, dtype=torch.uint8, device=dev)
         r_idx = torch.zeros(64, dtype=torch.int32, device=dev)
         r_cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+    alg1_tails = []
     handles, prepared = [], [[] for _ in range(n_rot)]
     prev_out = [None] * n_rot
     algo_bytes = 0
@@ -449,8 +450,13 @@ def main() -> int:
             kw = dict(R=R, B=w.B, seq_len=i32_dev(b["seq_len"]), kv_len=i32_dev(b["kv_len"]),
                       row_seq=i32_dev(b["row_seq"]), flags=args.flags, stream=stream)
             if alg1:
-                # run entry j of the model's batch reads row j of the pool; the live count is plan's, on device
-                kw = dict(R=w.B, B=w.B, n_rows_dev=state.run_count[hi], flags=args.flags, stream=stream)
+                # run entry j of the model's batch reads row j of the pool; the live count is plan's, on device;
+                # the call's own tail applies the decision block, the LLM's call also plans the next round
+                if len(alg1_tails) <= hi:
+                    alg1_tails.append(state.tail(hi, -1, spans=False, plan_next=(hi == 1), t_max=1 << 30,
+                                                 latency=lat_models))
+                kw = dict(R=w.B, B=w.B, n_rows_dev=state.run_count[hi], flags=args.flags, stream=stream,
+                          alg1_tail=alg1_tails[hi])
             elif hi == 1:
                 # batched step: the LLM head runs on the subset the SLM head routed, count on device
                 kw.update(row_idx=prev_out[i].llm_idx, n_rows_dev=prev_out[i].llm_count)
@@ -462,18 +468,17 @@ def main() -> int:
     rows_per_step = float(np.mean([b["R"] for b in heads[0]["batches"]]))
     decisions_per_step = rows_per_step            # rows decided by the first head of the step
 
+    if alg1:
+        # the first round's plans; every later round is planned by the LLM call of the round before
+        state.plan(0, 1 << 30, lat_models[0], stream=stream)
+        state.plan(1, 1 << 30, lat_models[1], stream=stream)
+
     def step(i):
         calls = prepared[i % n_rot]
-        if alg1:
-            state.plan(0, 1 << 30, lat_models[0], stream=stream)
-            state.plan(1, 1 << 30, lat_models[1], stream=stream)
         for call in calls:
             st = call.launch()
             if st != 0:
                 raise rs.RstitchError(st, "rstitch_route_ex")
-        if alg1:
-            for m in (0, 1):
-                state.commit(m, calls[m].out.tok, calls[m].out.mask, -1, spans=False, stream=stream)
         if with_router:
             o = calls[0].out
             router.forward(calls[0]._keep[1], 64, row_idx=o.llm_idx, n_rows_dev=o.llm_count, logits=r_logits,
@@ -484,7 +489,7 @@ def main() -> int:
         step(i)
     torch.cuda.synchronize()
     warm_launches = sum(rs.last_status(hd)["launches"] for hd in handles)     # also clears the counters
-    launches_per_step = warm_launches / float(Wm) + (4 if alg1 else 0) + (2 if with_router else 0)
+    launches_per_step = warm_launches / float(Wm) + (2 if with_router else 0)
 
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if dist is not None:
@@ -530,7 +535,7 @@ def main() -> int:
         dist.barrier()
     ms = ev0.elapsed_time(ev1)
     stats = [rs.last_status(hd) for hd in handles]
-    launches = sum(st["launches"] for st in stats) + (4 * K if alg1 else 0) + (2 * K if with_router else 0)
+    launches = sum(st["launches"] for st in stats) + (2 * K if with_router else 0)
     if graph is not None:
         launches = int(round(K * launches_per_step))      # replayed kernels are not counted by the handles
     if any(st["timeouts"] or st["nan_rows"] for st in stats):

@@ -98,6 +98,7 @@ typedef struct rstitch_handle_s *rstitch_handle_t;
  *               aligned; NULL uses the handle's own.  Two calls in flight at once on different
  *               streams must not share a workspace.
  */
+struct rstitch_alg1_tail_s;
 typedef struct rstitch_args_s {
     const void    *hidden;
     const void    *W_head;
@@ -122,6 +123,8 @@ typedef struct rstitch_args_s {
     float          temperature;     /* T_s > 0 */
     uint64_t       seed;            /* generator key */
     uint64_t       draw;            /* draw number: use a new one for every step */
+    /* optional (NULL: none): Algorithm 1's decision block run by this call itself, see rstitch_alg1_tail_t */
+    const struct rstitch_alg1_tail_s *alg1_tail;
 } rstitch_args_t;
 
 /* Device status word, accumulated since the handle was created or last read. */
@@ -258,6 +261,31 @@ int rstitch_alg1_plan(const rstitch_alg1_state_t *s, int B, int model, int t_max
 int rstitch_alg1_commit(const rstitch_alg1_state_t *s, int B, int model, const int32_t *run_idx,
                         const int32_t *run_count, const int32_t *row_off, const int32_t *tok,
                         const uint8_t *route_mask, int32_t eos_id, void *cuda_stream);
+
+/*
+ * The same steps without launches of their own: a routing call whose rstitch_args_t.alg1_tail points to one
+ * of these (a HOST structure, read during the call) goes on, in the block that has just written its tokens
+ * and mask, with the decision block of Algorithm 1 for the model's batch (exactly rstitch_alg1_commit with
+ * tok = tok_out and route_mask = route_mask of the call) and then, with plan_next != 0, with the planning of
+ * the next round for BOTH models (exactly rstitch_alg1_plan for model 0, then 1, writing the next_* arrays,
+ * which may be the buffers of the run lists just consumed).  A round of the loop is then two launches:
+ * the SLM head with {model 0, plan_next 0}, the LLM head with {model 1, plan_next 1}; only the first
+ * round's plans are calls of their own.  The routing call's rows are the model's batch: n_rows_dev =
+ * run_count, B at least the largest run count (without multi-row spans, row j belongs to run entry j and
+ * row_off is NULL).  Accepted by rstitch_route_ex and rstitch_shard_route.
+ */
+typedef struct rstitch_alg1_tail_s {
+    const rstitch_alg1_state_t *state;     /* HOST pointer to the structure of device arrays */
+    int32_t n_seq;                         /* sequences in the state */
+    int32_t model;                         /* 0 = SLM, 1 = LLM: whose batch this call decides */
+    const int32_t *run_idx, *run_count;    /* DEVICE: the model's run list from the last planning */
+    const int32_t *row_off;                /* DEVICE, optional: row offsets of the run entries' spans */
+    int32_t eos_id;
+    int32_t plan_next;                     /* non-zero: plan the next round for both models afterwards */
+    int32_t t_max;                         /* as in rstitch_alg1_plan (with plan_next) */
+    rstitch_latency_model_t latency[2];    /* Eq. 5 coefficients of model 0 and 1 (with plan_next) */
+    int32_t *next_run_idx[2], *next_run_count[2], *next_n_inf[2], *next_n_kv[2], *next_row_off[2];
+} rstitch_alg1_tail_t;
 
 /* ---- R-Stitch+ router ---------------------------------------------------------------------------- */
 

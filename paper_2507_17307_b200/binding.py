@@ -45,6 +45,7 @@ class _Args(C.Structure):
         ("llm_span", C.c_void_p), ("llm_row_off", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("temperature", C.c_float), ("seed", C.c_uint64), ("draw", C.c_uint64),
+        ("alg1_tail", C.c_void_p),
     ]
 
 
@@ -75,6 +76,15 @@ class _Alg1State(C.Structure):
     _fields_ = [("active", C.c_void_p), ("kv_slm", C.c_void_p), ("kv_llm", C.c_void_p), ("seq_len", C.c_void_p),
                 ("n_out", C.c_void_p), ("done", C.c_void_p), ("iters", C.c_void_p), ("kept", C.c_void_p),
                 ("steps", C.c_void_p), ("lat_ms", C.c_void_p), ("y", C.c_void_p), ("y_cap", C.c_int32)]
+
+
+class _Alg1Tail(C.Structure):
+    _fields_ = [("state", C.c_void_p), ("n_seq", C.c_int32), ("model", C.c_int32),
+                ("run_idx", C.c_void_p), ("run_count", C.c_void_p), ("row_off", C.c_void_p),
+                ("eos_id", C.c_int32), ("plan_next", C.c_int32), ("t_max", C.c_int32),
+                ("latency", LatencyModel * 2),
+                ("next_run_idx", C.c_void_p * 2), ("next_run_count", C.c_void_p * 2), ("next_n_inf", C.c_void_p * 2),
+                ("next_n_kv", C.c_void_p * 2), ("next_row_off", C.c_void_p * 2)]
 
 
 def library_path() -> str:
@@ -222,9 +232,10 @@ def route(hidden, W_head, tau: float, out: Optional[RouteOutputs] = None) -> Rou
 def route_ex(handle: Handle, hidden, W_head, tau: float, *, R: Optional[int] = None,
              B: Optional[int] = None, row_idx=None, row_seq=None, n_rows_dev=None, seq_len=None,
              kv_len=None, flags: int = 0, stream=None, out: Optional[RouteOutputs] = None,
-             workspace=None, check: bool = True, sample=None):
+             workspace=None, check: bool = True, sample=None, alg1_tail=None):
     """rstitch_route_ex.  Returns the outputs (or the status when check=False).
-    sample = (temperature, seed, draw) asks for a sampled token (RSTITCH_SAMPLE)."""
+    sample = (temperature, seed, draw) asks for a sampled token (RSTITCH_SAMPLE);
+    alg1_tail = Alg1State.tail(...) lets the call run Algorithm 1's decision block itself."""
     n_src, d = int(hidden.shape[0]), int(hidden.shape[1])
     V = int(W_head.shape[0])
     if R is None:
@@ -247,6 +258,8 @@ def route_ex(handle: Handle, hidden, W_head, tau: float, *, R: Optional[int] = N
     if sample is not None:
         a.flags |= SAMPLE
         a.temperature, a.seed, a.draw = float(sample[0]), int(sample[1]), int(sample[2])
+    if alg1_tail is not None:
+        a.alg1_tail = C.addressof(alg1_tail)
     st = lib().rstitch_route_ex(handle.ptr, C.byref(a), _stream_ptr(stream))
     if not check:
         return st
@@ -337,7 +350,7 @@ class PreparedCall:
 
     def __init__(self, handle: Handle, hidden, W_head, tau: float, out: RouteOutputs, *, R=None, B=None,
                  row_idx=None, row_seq=None, n_rows_dev=None, seq_len=None, kv_len=None, flags=0,
-                 stream=None):
+                 stream=None, alg1_tail=None):
         n_src, d = int(hidden.shape[0]), int(hidden.shape[1])
         if R is None:
             R = int(row_idx.shape[0]) if row_idx is not None else n_src
@@ -352,7 +365,9 @@ class PreparedCall:
         a.tok_out, a.ent_out, a.route_mask = _ptr(out.tok), _ptr(out.ent), _ptr(out.mask)
         a.llm_idx, a.llm_count = _ptr(out.llm_idx), _ptr(out.llm_count)
         a.llm_span, a.llm_row_off = _ptr(out.llm_span), _ptr(out.llm_row_off)
-        self._keep = (handle, hidden, W_head, out, row_idx, row_seq, n_rows_dev, seq_len, kv_len)
+        if alg1_tail is not None:
+            a.alg1_tail = C.addressof(alg1_tail)
+        self._keep = (handle, hidden, W_head, out, row_idx, row_seq, n_rows_dev, seq_len, kv_len, alg1_tail)
         self._args = a
         self._ref = C.byref(a)
         self._h = handle.ptr
@@ -493,6 +508,27 @@ class Alg1State:
                                      _ptr(self.n_kv[model]), _ptr(self.row_off[model]), _stream_ptr(stream))
         if st != 0:
             raise RstitchError(st, "rstitch_alg1_plan")
+
+    def tail(self, model: int, eos_id: int, spans: bool = True, plan_next: bool = False, t_max: int = 0,
+             latency=None):
+        """rstitch_alg1_tail_t for a routing call on `model`'s batch (pass it as alg1_tail=): the call
+        then applies the decision block to plan(model)'s run list itself and, with plan_next, plans the
+        next round for both models (latency = the two models' LatencyModel) into this object's run lists.
+        Keep the returned structure alive while calls that use it may still be issued."""
+        t = _Alg1Tail()
+        t.state = C.addressof(self._c)
+        t.n_seq, t.model, t.eos_id = self.B, int(model), int(eos_id)
+        t.run_idx, t.run_count = _ptr(self.run_idx[model]), _ptr(self.run_count[model])
+        t.row_off = _ptr(self.row_off[model]) if spans else None
+        t.plan_next, t.t_max = int(bool(plan_next)), int(t_max)
+        if plan_next:
+            for m in (0, 1):
+                t.latency[m] = latency[m]
+                t.next_run_idx[m], t.next_run_count[m] = _ptr(self.run_idx[m]), _ptr(self.run_count[m])
+                t.next_n_inf[m], t.next_n_kv[m] = _ptr(self.n_inf[m]), _ptr(self.n_kv[m])
+                t.next_row_off[m] = _ptr(self.row_off[m])
+        t._keep = self
+        return t
 
     def commit(self, model: int, tok, mask, eos_id: int, spans: bool = True, stream=None):
         """Applies the decision block to the run list of plan(model).  spans=True: tok has one entry

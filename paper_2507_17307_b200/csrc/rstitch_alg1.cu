@@ -7,8 +7,8 @@
 //   commit: the decision block after the entropy test -- discard and roll back on an SLM hand-off,
 //           hand back from the LLM on low entropy, append the token, stop on EOS.
 // Integer work on B elements; one block, warp ballots and prefix sums for the ordered run list.
-#include "../../include/rstitch.h"
-#include <cuda_runtime.h>
+#include "rstitch_alg1.cuh"
+#include "rstitch_kernels.cuh"
 
 #include <cmath>
 
@@ -28,89 +28,29 @@ alg1_init_kernel(rstitch_alg1_state_t s, int B, const int32_t *prompt_len)
     }
 }
 
-// One block.  Sequences are taken in chunks of blockDim.x; inside a chunk a ballot gives each selected
-// sequence its rank within the warp, warp totals are scanned in shared memory and a carry links the
-// chunks, so run_idx comes out ascending and row_off is the exclusive scan of n_inf in that order.
+// One block: see alg1_plan_block.
 __global__ void __launch_bounds__(kThreads)
 alg1_plan_kernel(rstitch_alg1_state_t s, int B, int model, int t_max, rstitch_latency_model_t lat,
                  int32_t *run_idx, int32_t *run_count, int32_t *n_inf_out, int32_t *n_kv_out, int32_t *row_off)
 {
-    __shared__ int w_cnt[kThreads / 32], w_rows[kThreads / 32], carry[2];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    int32_t *kv = model == 0 ? s.kv_slm : s.kv_llm;
-    if (threadIdx.x == 0) { carry[0] = 0; carry[1] = 0; }
-    __syncthreads();
-    for (int base = 0; base < B; base += blockDim.x) {
-        const int b = base + threadIdx.x;
-        bool run = false;
-        int n_inf = 0, n_kv = 0;
-        if (b < B) run = !s.done[b] && s.iters[b] < t_max && s.active[b] == model;   // "for t = 1 .. T_max"
-        if (run) {
-            const int L = kv[b], len = s.seq_len[b];
-            n_kv = L;
-            if (L < len) { n_inf = len - L; kv[b] = len + 1; }         // prefill of the missing span
-            else         { n_inf = 1;       kv[b] = L + 1; }           // decode
-            const double ni = (double)n_inf, nk = (double)n_kv;
-            s.lat_ms[b] += lat.a * ni * nk + lat.b * ni * ni + lat.c * ni + lat.d;     // Eq. 5
-            s.steps[model * B + b] += 1;
-            s.iters[b] += 1;
-        }
-        const unsigned ball = __ballot_sync(0xffffffffu, run);
-        const int rank = __popc(ball & ((1u << lane) - 1u));
-        int incl = n_inf;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) { w_cnt[warp] = __popc(ball); w_rows[warp] = incl; }
-        __syncthreads();
-        int pre_cnt = carry[0], pre_rows = carry[1];
-        for (int w = 0; w < warp; ++w) { pre_cnt += w_cnt[w]; pre_rows += w_rows[w]; }
-        if (run) {
-            const int j = pre_cnt + rank;
-            run_idx[j] = b;
-            n_inf_out[j] = n_inf;
-            n_kv_out[j] = n_kv;
-            row_off[j] = pre_rows + incl - n_inf;
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            int c = 0, r = 0;
-            for (int w = 0; w < nwarps; ++w) { c += w_cnt[w]; r += w_rows[w]; }
-            carry[0] += c; carry[1] += r;
-        }
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) { *run_count = carry[0]; row_off[carry[0]] = carry[1]; }
+    __shared__ int smem[34];
+    rstitch::alg1_plan_block(s, B, model, t_max, lat, run_idx, run_count, n_inf_out, n_kv_out, row_off, smem);
 }
 
 __global__ void __launch_bounds__(kThreads)
 alg1_commit_kernel(rstitch_alg1_state_t s, int B, int model, const int32_t *run_idx, const int32_t *run_count,
                    const int32_t *row_off, const int32_t *tok, const uint8_t *mask, int32_t eos_id)
 {
-    const int n = *run_count;
-    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x) {
-        const int b = run_idx[j];
-        if (b < 0 || b >= B) continue;
-        const int row = row_off ? row_off[j + 1] - 1 : j;      // a prefill yields its token at the end of the span
-        const int32_t yt = tok[row];
-        if (mask[j]) {                                         // H_t > tau
-            if (model == 0) {                                  // SLM -> LLM: discard, roll the cache back
-                s.kv_slm[b] -= 1;
-                s.active[b] = 1;
-                continue;
-            }                                                  // on the LLM: keep decoding with it
-        } else if (model == 1) {
-            s.active[b] = 0;                                   // LLM -> SLM
-        }
-        const int k = s.n_out[b];
-        if (k < s.y_cap) s.y[(size_t)b * s.y_cap + k] = yt;    // append y_t
-        s.n_out[b] = k + 1;
-        s.seq_len[b] += 1;
-        s.kept[model * B + b] += 1;
-        if (yt == eos_id) s.done[b] = 1;
-    }
+    rstitch::alg1_commit_entries(s, B, model, run_idx, *run_count, row_off, tok, mask, eos_id,
+                                 (int)(blockIdx.x * blockDim.x + threadIdx.x), (int)(gridDim.x * blockDim.x));
+}
+
+// The block a routing call would have run after its own tail, for a call that has no rows to evaluate.
+__global__ void __launch_bounds__(kThreads)
+alg1_tail_kernel(rstitch::Alg1Tail a, const int32_t *tok, const uint8_t *mask)
+{
+    __shared__ int smem[34];
+    rstitch::alg1_tail_block(a, tok, mask, smem);
 }
 
 bool state_ok(const rstitch_alg1_state_t *s)
@@ -120,6 +60,18 @@ bool state_ok(const rstitch_alg1_state_t *s)
 }
 
 }  // namespace
+
+namespace rstitch {
+
+bool alg1_state_ok(const rstitch_alg1_state_t *s) { return state_ok(s); }
+
+cudaError_t launch_alg1_tail(const Alg1Tail &a, const int32_t *tok, const uint8_t *mask, cudaStream_t stream)
+{
+    alg1_tail_kernel<<<1, kThreads, 0, stream>>>(a, tok, mask);
+    return cudaGetLastError();
+}
+
+}  // namespace rstitch
 
 extern "C" {
 

@@ -185,17 +185,56 @@ bool use_umma(int R, int d, int V, uint32_t flags)
     return R > kGemvMaxRows;
 }
 
+// rstitch_alg1_tail_t (host) -> the device copy the tails carry; false: a bad structure.
+bool make_alg1_tail(const rstitch_alg1_tail_t *t, Alg1Tail *out)
+{
+    out->on = 0;
+    if (!t) return true;
+    if (!alg1_state_ok(t->state) || t->n_seq < 0 || (t->model != 0 && t->model != 1) || !t->run_count ||
+        (t->n_seq > 0 && !t->run_idx))
+        return false;
+    out->on = 1;
+    out->s = *t->state;
+    out->n_seq = t->n_seq; out->model = t->model;
+    out->run_idx = t->run_idx; out->run_count = t->run_count; out->row_off = t->row_off;
+    out->eos_id = t->eos_id; out->plan_next = t->plan_next ? 1 : 0; out->t_max = t->t_max;
+    for (int m = 0; m < 2; ++m) {
+        out->lat[m] = t->latency[m];
+        out->nx_idx[m] = t->next_run_idx[m]; out->nx_cnt[m] = t->next_run_count[m];
+        out->nx_ninf[m] = t->next_n_inf[m]; out->nx_nkv[m] = t->next_n_kv[m]; out->nx_off[m] = t->next_row_off[m];
+        if (t->plan_next) {
+            if (t->t_max < 0 || !out->nx_cnt[m] || !out->nx_off[m]) return false;
+            if (t->n_seq > 0 && (!out->nx_idx[m] || !out->nx_ninf[m] || !out->nx_nkv[m])) return false;
+            if (!std::isfinite(t->latency[m].a) || !std::isfinite(t->latency[m].b) ||
+                !std::isfinite(t->latency[m].c) || !std::isfinite(t->latency[m].d))
+                return false;
+        }
+    }
+    return true;
+}
+
 // Validated arguments -> kernels.  With shard_stats the head is a vocabulary shard starting at entry
 // v_base: per-row statistics go to shard_stats and no routing output is touched.
 int enqueue_head(rstitch_handle_s *h, const rstitch_args_t *a, cudaStream_t stream, float *shard_stats,
                         int v_base)
 {
+    Alg1Tail alg1;
+    if (!make_alg1_tail(shard_stats ? nullptr : a->alg1_tail, &alg1)) return RSTITCH_ERR_INVALID_ARG;
     if (!shard_stats && (a->R == 0 || a->B == 0)) {
         // nothing to evaluate or nothing to decide: the compaction of an empty mask
         if (cudaMemsetAsync(a->llm_count, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
         if (a->seq_len && a->llm_row_off &&
             cudaMemsetAsync(a->llm_row_off, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
-        if (a->R == 0) return RSTITCH_OK;
+        if (a->R == 0) {
+            if (alg1.on) {                 // no rows, but the loop goes on: the block on its own
+                if (launch_alg1_tail(alg1, a->tok_out, a->route_mask, stream) != cudaSuccess) {
+                    cudaGetLastError();
+                    return RSTITCH_ERR_CUDA;
+                }
+                h->launch_count += 1;
+            }
+            return RSTITCH_OK;
+        }
     }
 
     HeadArgs ha;
@@ -220,6 +259,7 @@ int enqueue_head(rstitch_handle_s *h, const rstitch_args_t *a, cudaStream_t stre
     ta.llm_span = a->llm_span; ta.llm_row_off = a->llm_row_off;
     ta.stat = h->stat;
     ta.shard_stats = shard_stats; ta.v_base = v_base;
+    ta.alg1 = alg1;
 
     void *ws = a->workspace ? a->workspace : h->ws;
     Scratch sc = scratch_carve(ws);
@@ -330,11 +370,22 @@ int rstitch_shard_route(rstitch_handle_t h, const rstitch_args_t *a, const void 
     if (!aligned(gathered, 4)) return RSTITCH_ERR_BAD_ALIGN;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     h->last_stream = stream;
+    Alg1Tail alg1;
+    if (!make_alg1_tail(a->alg1_tail, &alg1)) return RSTITCH_ERR_INVALID_ARG;
     if (a->R == 0 || a->B == 0) {
         if (cudaMemsetAsync(a->llm_count, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
         if (a->seq_len && a->llm_row_off &&
             cudaMemsetAsync(a->llm_row_off, 0, sizeof(int32_t), stream) != cudaSuccess) return RSTITCH_ERR_CUDA;
-        if (a->R == 0) return RSTITCH_OK;
+        if (a->R == 0) {
+            if (alg1.on) {
+                if (launch_alg1_tail(alg1, a->tok_out, a->route_mask, stream) != cudaSuccess) {
+                    cudaGetLastError();
+                    return RSTITCH_ERR_CUDA;
+                }
+                h->launch_count += 1;
+            }
+            return RSTITCH_OK;
+        }
     }
     TailArgs ta;
     ta.R = a->R; ta.B = a->B; ta.V = a->V;
@@ -345,6 +396,7 @@ int rstitch_shard_route(rstitch_handle_t h, const rstitch_args_t *a, const void 
     ta.llm_span = a->llm_span; ta.llm_row_off = a->llm_row_off;
     ta.stat = h->stat;
     ta.shard_stats = nullptr; ta.v_base = 0;
+    ta.alg1 = alg1;
     Scratch sc = scratch_carve(h->ws);
     int launched = 0;
     cudaError_t e = launch_shard_merge((const float *)gathered, n_shards, a->n_rows_dev, ta, sc.ticket, stream,

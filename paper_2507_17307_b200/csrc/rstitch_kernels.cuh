@@ -48,6 +48,11 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
 cudaError_t launch_shard_merge(const float *gathered, int n_shards, const int32_t *n_rows_dev, const TailArgs &t,
                                unsigned *ticket, cudaStream_t stream, int *launched);
 
+// Algorithm 1's block after a routing call that has no rows of its own (one small launch), and the
+// check of a caller's state structure.
+bool        alg1_state_ok(const rstitch_alg1_state_t *s);
+cudaError_t launch_alg1_tail(const Alg1Tail &a, const int32_t *tok, const uint8_t *mask, cudaStream_t stream);
+
 // Upper bound on the partials per row of any kernel for a vocabulary of V rows.
 __host__ __device__ inline size_t max_slices_for(int V)
 {

@@ -92,6 +92,7 @@ extern "C" int rstitch_route_static(const void *hidden, const void *W_head, int 
     ta.llm_idx = llm_idx; ta.llm_count = llm_count; ta.llm_span = nullptr; ta.llm_row_off = nullptr;
     ta.stat = (DevStat *)((char *)base + kStatOffset);
     ta.shard_stats = nullptr; ta.v_base = 0;
+    ta.alg1.on = 0;
     Scratch sc = scratch_carve(base);
     cudaError_t e = launch_head_gemv(ha, ta, sc, sms, stream);
     if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }

@@ -4,6 +4,7 @@
 #pragma once
 #include "rstitch_stats.cuh"
 #include "rstitch_ptx.cuh"
+#include "rstitch_alg1.cuh"
 #include <stdint.h>
 
 namespace rstitch {
@@ -68,6 +69,7 @@ struct TailArgs {
     // index of the best entry) and nothing is decided: shard_merge_kernel does that on the gathered shards.
     float   *shard_stats;        // [R][5] or nullptr
     int      v_base;
+    Alg1Tail alg1;               // optional: Algorithm 1's decision block (and the next round's plans) after S6
 };
 
 constexpr int kShardWords = 5;
@@ -393,10 +395,14 @@ __device__ inline void tail_route_warp(const TailArgs &a)
 __device__ inline void tail_route(const TailArgs &a, int *smem)
 {
     if (a.shard_stats) return;                       // a vocabulary shard decides nothing
-    if (a.B <= 32 && a.row_seq == nullptr) { tail_route_warp(a); return; }
-    tail_mask(a);
-    tail_compact(a.route_mask, a.B, a.seq_len, a.kv_len, a.llm_idx, a.llm_count, a.llm_span,
-                 a.llm_row_off, a.stat, smem);
+    if (a.B <= 32 && a.row_seq == nullptr) {
+        tail_route_warp(a);
+    } else {
+        tail_mask(a);
+        tail_compact(a.route_mask, a.B, a.seq_len, a.kv_len, a.llm_idx, a.llm_count, a.llm_span,
+                     a.llm_row_off, a.stat, smem);
+    }
+    if (a.alg1.on) alg1_tail_block(a.alg1, a.tok_out, a.route_mask, smem);
 }
 
 }  // namespace rstitch

@@ -96,8 +96,11 @@ def test_recorded_streams(rs, oracle, B, T, seed):
         assert np.array_equal(got[k], again[k]), k
 
 
-def test_end_to_end_with_the_routing_decision(rs, oracle):
-    # two small heads; the tokens and masks come from rstitch_route_ex on the model's batch of rows
+@pytest.mark.parametrize("fused", [False, True])
+def test_end_to_end_with_the_routing_decision(rs, oracle, fused):
+    # two small heads; the tokens and masks come from rstitch_route_ex on the model's batch of rows.
+    # fused: no commit launches and only the first round's plans -- the routing calls carry the decision
+    # block in their own tail (alg1_tail), the LLM's call also the next round's planning
     import torch
     B, T, tau, eos = 16, 10, 0.3, -1
     c = coeffs()
@@ -123,12 +126,20 @@ def test_end_to_end_with_the_routing_decision(rs, oracle):
     prompt = rng.integers(1, 9, size=B).astype(np.int32)        # short prompts keep the spans small
     st = rs.Alg1State(B, y_cap=T)
     st.init(to_dev_i32(prompt))
+    tails = [st.tail(0, eos), st.tail(1, eos, plan_next=True, t_max=T, latency=lat)]
+    empty_calls = 0
     for t in range(T):
+        if not fused or t == 0:
+            for m in (0, 1):
+                st.plan(m, T, lat[m])
+        counts = [int(st.run_count[m].item()) for m in (0, 1)]      # both read before the LLM call replans
         for m in (0, 1):
-            st.plan(m, T, lat[m])
-        for m in (0, 1):
-            n = int(st.run_count[m].item())
+            n = counts[m]
             if n == 0:
+                if fused:      # no rows, but the loop goes on: the call runs the block on its own
+                    rs.route_ex(handle, torch.zeros((0, 64), dtype=torch.bfloat16, device="cuda"), w_dev[m], tau,
+                                R=0, B=0, alg1_tail=tails[m])
+                    empty_calls += 1
                 continue
             idx = st.run_idx[m].cpu().numpy()[:n]
             off = st.row_off[m].cpu().numpy()[:n + 1]
@@ -136,8 +147,10 @@ def test_end_to_end_with_the_routing_decision(rs, oracle):
             rows = gen.f32_to_bf16_bits(rng.standard_normal((R, 64)).astype(np.float32))   # span filler rows
             rows[off[1:] - 1] = hid[m][idx, t]                                            # span ends: the real step
             row_seq = np.repeat(np.arange(n, dtype=np.int32), np.diff(off))
-            out = rs.route_ex(handle, to_dev_bf16(rows), w_dev[m], tau, R=R, B=n, row_seq=to_dev_i32(row_seq))
-            st.commit(m, out.tok, out.mask, eos)
+            out = rs.route_ex(handle, to_dev_bf16(rows), w_dev[m], tau, R=R, B=n, row_seq=to_dev_i32(row_seq),
+                              alg1_tail=tails[m] if fused else None)
+            if not fused:
+                st.commit(m, out.tok, out.mask, eos)
             seen = out.tok.cpu().numpy()[off[1:] - 1]
             exact = ~tie[m][idx, t]
             assert np.array_equal(seen[exact], tok[m][idx, t][exact])
@@ -152,6 +165,52 @@ def test_end_to_end_with_the_routing_decision(rs, oracle):
         routed_any |= ref["steps_llm"] > 0
     assert routed_any, "the workload never handed a step to the LLM"
     assert rs.last_status(handle)["timeouts"] == 0
+    assert not fused or empty_calls > 0, "the stand-alone form of the block never ran"
+    handle.destroy()
+
+
+def test_fused_tail_on_both_kernel_families_and_bad_structures(rs, oracle):
+    # one round on a single-row-per-entry batch through each head kernel, against plan + call + commit
+    import torch
+    B, tau, eos = 40, 0.3, 3
+    c = coeffs()
+    lat = [rs.LatencyModel(*c["SLM-1.5B"]), rs.LatencyModel(*c["LLM-7B"])]
+    w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=256, V=2053, seed=8300)
+    w_bits = gen.make_w_head(w)
+    w_dev, hid = to_dev_bf16(w_bits), to_dev_bf16(gen.make_hidden(w, w_bits, 0)[0])
+    prompt = to_dev_i32(np.arange(5, 5 + B))
+    handle = rs.Handle(512, 256, 4096)
+    for flags in (rs.PATH_GEMV, rs.PATH_UMMA):
+        ref_st, st = rs.Alg1State(B, y_cap=4), rs.Alg1State(B, y_cap=4)
+        for s_ in (ref_st, st):
+            s_.init(prompt)
+            s_.plan(0, 9, lat[0])
+            s_.plan(1, 9, lat[1])
+        out = rs.route_ex(handle, hid, w_dev, tau, n_rows_dev=ref_st.run_count[0], flags=flags)
+        ref_st.commit(0, out.tok, out.mask, eos, spans=False)
+        ref_st.plan(0, 9, lat[0])
+        ref_st.plan(1, 9, lat[1])
+        tail = st.tail(0, eos, spans=False, plan_next=True, t_max=9, latency=lat)
+        rs.route_ex(handle, hid, w_dev, tau, n_rows_dev=st.run_count[0], flags=flags, alg1_tail=tail)
+        torch.cuda.synchronize()
+        a, b = state_to_host(ref_st), state_to_host(st)
+        for k in a:
+            assert np.array_equal(a[k], b[k]), (flags, k)
+        for m in (0, 1):
+            n = int(ref_st.run_count[m].item())
+            assert n == int(st.run_count[m].item()) and (m == 0 or n > 0)
+            assert torch.equal(ref_st.run_idx[m][:n], st.run_idx[m][:n])
+            assert torch.equal(ref_st.row_off[m][:n + 1], st.row_off[m][:n + 1])
+            assert torch.equal(ref_st.n_inf[m][:n], st.n_inf[m][:n]) and torch.equal(ref_st.n_kv[m][:n], st.n_kv[m][:n])
+    bad = st.tail(0, eos)
+    bad.model = 2
+    assert rs.route_ex(handle, hid, w_dev, tau, alg1_tail=bad, check=False) == -1
+    bad = st.tail(1, eos, plan_next=True, t_max=9, latency=lat)
+    bad.next_row_off[1] = None
+    assert rs.route_ex(handle, hid, w_dev, tau, alg1_tail=bad, check=False) == -1
+    bad = st.tail(0, eos)
+    bad.run_count = None
+    assert rs.route_ex(handle, hid, w_dev, tau, alg1_tail=bad, check=False) == -1
     handle.destroy()
 
 
