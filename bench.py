@@ -133,14 +133,14 @@ def measured_peaks() -> dict:
 # once any of them has changed the counters no longer describe the kernel and the figure reads null.
 NCU_TRAFFIC = {
     "c2_slm_b1":
-    {"bytes": 471029248, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
-     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "d5767ba87bc635bf71f9069bcd7b408ff46f8339a455a5ff627f7a6bec3cbdb6", "rstitch_tail.cuh": "c7354c820b08678c99a76fe9f95332a64ac1a839c76083648825f9da6ec8ad71", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 471142400, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
+     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "0f73425c4cb67810f1adb034f8e18534119ded82a547f9cf295d8c52e9fd561f", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
     "c4_slm_b64":
-    {"bytes": 471211008, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
-     "sources": {"rstitch_umma.cu": "95c15fe676ede5ff8503be2afab0782f79839b0f0a88734d0bec3a0ae4a4bba9", "rstitch_kernels.cuh": "d5767ba87bc635bf71f9069bcd7b408ff46f8339a455a5ff627f7a6bec3cbdb6", "rstitch_tail.cuh": "c7354c820b08678c99a76fe9f95332a64ac1a839c76083648825f9da6ec8ad71", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 471890176, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
+     "sources": {"rstitch_umma.cu": "44e4753e7db25c6c2bd1eb75550c6565b60f03e0f6112c88ce7063728df15ded", "rstitch_kernels.cuh": "0f73425c4cb67810f1adb034f8e18534119ded82a547f9cf295d8c52e9fd561f", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
     "c5_catchup":
-    {"bytes": 1668683672, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
-     "sources": {"rstitch_umma.cu": "95c15fe676ede5ff8503be2afab0782f79839b0f0a88734d0bec3a0ae4a4bba9", "rstitch_kernels.cuh": "d5767ba87bc635bf71f9069bcd7b408ff46f8339a455a5ff627f7a6bec3cbdb6", "rstitch_tail.cuh": "c7354c820b08678c99a76fe9f95332a64ac1a839c76083648825f9da6ec8ad71", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 1673879808, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
+     "sources": {"rstitch_umma.cu": "44e4753e7db25c6c2bd1eb75550c6565b60f03e0f6112c88ce7063728df15ded", "rstitch_kernels.cuh": "0f73425c4cb67810f1adb034f8e18534119ded82a547f9cf295d8c52e9fd561f", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
 }
 
 
