@@ -371,6 +371,16 @@ int rstitch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, vo
  * Returns RSTITCH_ERR_TIMEOUT if a bounded wait gave up since the last read. */
 int rstitch_last_status(rstitch_handle_t h, rstitch_devstat_t *out);
 
+/*
+ * Self-test of the error path of the kernels' bounded waits (every wait on a copy or on the tensor pipe
+ * gives up after a cycle limit instead of hanging): enqueues one tiny kernel whose only wait can never be
+ * satisfied and is limited to about a millisecond.  It gives up, records that in the status word like any
+ * other wait and returns; the next rstitch_last_status(h, ...) returns RSTITCH_ERR_TIMEOUT with
+ * timeouts = 1 and timeout_site = RSTITCH_SELFTEST_SITE, and the handle and the context stay usable.
+ */
+#define RSTITCH_SELFTEST_SITE 0x7e57u
+int rstitch_selftest_wait(rstitch_handle_t h, void *cuda_stream);
+
 /* Static, never NULL. */
 const char *rstitch_status_string(int status);
 

@@ -125,6 +125,8 @@ def lib():
         L.rstitch_path_name.restype = C.c_char_p
         L.rstitch_route_static.argtypes = [vp, vp, i, i, i, f, vp, vp, vp, vp, vp, vp]
         L.rstitch_route_static.restype = i
+        L.rstitch_selftest_wait.argtypes = [vp, vp]
+        L.rstitch_selftest_wait.restype = i
         L.rstitch_shard_stats.argtypes = [vp, C.POINTER(_Args), C.c_int32, vp, vp]
         L.rstitch_shard_stats.restype = i
         L.rstitch_shard_route.argtypes = [vp, C.POINTER(_Args), vp, C.c_int32, vp]
@@ -455,6 +457,15 @@ def compact(mask, idx=None, count=None, stream=None):
     if st != 0:
         raise RstitchError(st, "rstitch_compact")
     return idx, count
+
+
+SELFTEST_SITE = 0x7E57
+
+
+def selftest_wait(handle: Handle, stream=None) -> int:
+    """rstitch_selftest_wait: makes one bounded device-side wait run out (about a millisecond); the next
+    last_status(handle) reports the timeout."""
+    return lib().rstitch_selftest_wait(handle.ptr, _stream_ptr(stream))
 
 
 def last_status(handle: Optional[Handle] = None) -> dict:

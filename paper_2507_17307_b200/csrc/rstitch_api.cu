@@ -577,6 +577,17 @@ int rstitch_compact(const uint8_t *mask, int B, int32_t *idx, int32_t *count, vo
     return RSTITCH_OK;
 }
 
+int rstitch_selftest_wait(rstitch_handle_t h, void *cuda_stream)
+{
+    if (!h) return RSTITCH_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    h->last_stream = stream;
+    // ~1 ms at the top SM clock: long enough to be a real wait, far below anything a watchdog minds
+    if (launch_wait_selftest(h->stat, 2000000ll, stream) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+    h->launch_count += 1;
+    return RSTITCH_OK;
+}
+
 int rstitch_last_status(rstitch_handle_t h, rstitch_devstat_t *out)
 {
     if (!out) return RSTITCH_ERR_INVALID_ARG;

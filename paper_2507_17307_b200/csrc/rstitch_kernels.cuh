@@ -53,6 +53,10 @@ cudaError_t launch_shard_merge(const float *gathered, int n_shards, const int32_
 bool        alg1_state_ok(const rstitch_alg1_state_t *s);
 cudaError_t launch_alg1_tail(const Alg1Tail &a, const int32_t *tok, const uint8_t *mask, cudaStream_t stream);
 
+// The bounded wait running out on purpose (rstitch_selftest_wait): site id it leaves in the status word.
+constexpr unsigned kSelftestSite = 0x7e57u;
+cudaError_t launch_wait_selftest(DevStat *stat, long long limit_cycles, cudaStream_t stream);
+
 // Upper bound on the partials per row of any kernel for a vocabulary of V rows.
 __host__ __device__ inline size_t max_slices_for(int V)
 {

@@ -61,7 +61,8 @@ constexpr long long kWaitLimitCycles = 1ll << 32;
 
 // Waits until the phase with the given parity has completed.  Gives up when the cycle limit
 // runs out or another thread of the block has raised *abort_flag; returns false then.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          long long limit_cycles = kWaitLimitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -69,7 +70,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) return false;
+            if (clock64() - t0 > limit_cycles) return false;
         }
     }
 }

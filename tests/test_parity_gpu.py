@@ -468,3 +468,21 @@ def test_maximum_sizes(rs, oracle, B, d, V, path):
     finally:
         h.destroy()
     assert rs.workspace_bytes(16385, 64, 512) == 0 and rs.workspace_bytes(4, 16392, 512) == 0
+
+
+def test_bounded_wait_runs_out_and_the_handle_stays_usable(rs, handle, oracle):
+    # every device-side wait in the kernels has a cycle limit; this makes one run out (a barrier nothing
+    # arrives at, limited to ~1 ms) and checks the report, then that the same handle still decides correctly
+    import time
+    import torch
+    rs.last_status(handle)
+    t0 = time.perf_counter()
+    assert rs.selftest_wait(handle) == 0
+    st = rs.last_status(handle)
+    assert time.perf_counter() - t0 < 1.0
+    assert st["status"] == -6 and st["timeouts"] == 1 and st["timeout_site"] == rs.SELFTEST_SITE
+    assert rs.status_string(-6) == "device-side wait timed out"
+    w = gen.scaled(gen.WORKLOADS["c3_llm_b4"], V=6007, d=512)
+    for flags in (rs.PATH_GEMV, rs.PATH_UMMA):
+        check_case(rs, handle, oracle, w, [0], flags=flags)          # asserts a clean status word again
+    assert torch.cuda.is_available()
