@@ -37,7 +37,11 @@ constexpr int kMaxRows = 16384;
 
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-constexpr int kGemvMaxRows = 1;      // with 4 rows the CUDA-core kernel already falls to ~74 % of HBM; the tensor-core kernel holds ~87 %
+// Rows up to which the CUDA-core streaming kernel is taken.  Measured on the 3584 x 152064 head (us per call):
+//   rows       1      2      3      4      8
+//   streaming  160    175    211    228    453     (contiguous bulk copies: the best DRAM pattern, FMA-bound from 3 rows)
+//   tcgen05    173    179    176    178    184     (128-byte pieces of many rows per copy: ~7 % slower streaming)
+constexpr int kGemvMaxRows = 2;
 
 size_t ws_partials_bytes(int R, int V)
 {
