@@ -32,6 +32,10 @@ constexpr int kProducers = 1;                        // copy-issuing warps.  One
                                                      // microsecond and separate warps issue in parallel (a probe reached
                                                      // 19/us with four), but these kernels need at most ~6/us and measured
                                                      // the same with 1, 2 and 3; the dealing code below stays general
+// k-steps whose copies the one-M-tile kernel issues together.  Measured on the 3584 x 152064 head with 16
+// rows: 1 -> 197 us, 2 -> 181 us, 4 -> 200 us (a group needs that many free stages at once; with eight
+// stages a group of four leaves too little in flight).
+constexpr int kIssueGroup = 2;
 constexpr int kEpiWarps  = 8;
 constexpr int kThreads   = 64 + kEpiWarps * 32;      // head_umma_kernel: producer, MMA, 8 epilogue warps
 constexpr int kMaxStages = 8;
@@ -244,32 +248,46 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
             bool live = true;
             for (int j = 0; live && j < sch.n_items; ++j) {
                 const Item it = sch.item(j);
-                for (int ks = 0; ks < nK; ++ks) {
-                    if (!ptx::mbar_wait(ptx::smem_u32(&s_empty[stage]), (uint32_t)((round & 1) ^ 1), &s_abort)) {
-                        if (!s_abort) raise_abort(&s_abort, t.stat, 0x201u);
-                        live = false;
-                        break;
+                const uint32_t bytes = (uint32_t)((plan.a_rows + it.N) * kTileK * 2);
+                // The k-steps are issued in groups: a copy brings 128 bytes of each of its rows, so the
+                // copies of kIssueGroup consecutive k-steps, issued back to back box by box, ask DRAM for
+                // kIssueGroup * 128 contiguous bytes of a row at a time instead of 128.
+                for (int ks = 0; live && ks < nK; ks += kIssueGroup) {
+                    int ng = nK - ks < kIssueGroup ? nK - ks : kIssueGroup;
+                    if (ng > n_stages) ng = n_stages;
+                    uint32_t full[kIssueGroup], a_dst[kIssueGroup];
+                    for (int g = 0; g < ng; ++g) {
+                        int sg = stage + g, rd = round;
+                        if (sg >= n_stages) { sg -= n_stages; ++rd; }
+                        if (!ptx::mbar_wait(ptx::smem_u32(&s_empty[sg]), (uint32_t)((rd & 1) ^ 1), &s_abort)) {
+                            if (!s_abort) raise_abort(&s_abort, t.stat, 0x201u);
+                            live = false;
+                            ng = g;                  // the stages armed so far still get their copies
+                            break;
+                        }
+                        full[g] = ptx::smem_u32(&s_full[sg]);
+                        a_dst[g] = ring + (uint32_t)(sg * plan.stage_bytes);
+                        ptx::mbar_arrive_expect_tx(full[g], bytes);
                     }
-                    const uint32_t full = ptx::smem_u32(&s_full[stage]);
-                    const uint32_t a_dst = ring + (uint32_t)(stage * plan.stage_bytes);
-                    const uint32_t b_dst = a_dst + (uint32_t)plan.a_bytes;
                     // only the first a_rows rows of the hidden tile are fetched; the MMA reads all 128,
                     // and what the stale rows produce lands in accumulator rows nobody looks at
-                    if (pid == 0) {
-                        ptx::mbar_arrive_expect_tx(full, (uint32_t)((plan.a_rows + it.N) * kTileK * 2));
-                        ptx::tma_g2s_2d(a_dst, &tm_hidden, ks * kTileK, 0, full);
-                    }
+                    for (int g = 0; g < ng; ++g)
+                        ptx::tma_g2s_2d(a_dst[g], &tm_hidden, (ks + g) * kTileK, 0, full[g]);
                     int r = 0;
 #pragma unroll
                     for (int b = 4; b >= 0; --b) {
                         const int rows = 16 << b;
                         if (it.N - r >= rows) {
-                            ptx::tma_g2s_2d(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK, it.v0 + r, full);
+                            for (int g = 0; g < ng; ++g)
+                                ptx::tma_g2s_2d(a_dst[g] + (uint32_t)plan.a_bytes + (uint32_t)r * 128u, &tm_w.box[b],
+                                                (ks + g) * kTileK, it.v0 + r, full[g]);
                             r += rows;
                         }
                     }
-                    ++issued;
-                    if (++stage == n_stages) { stage = 0; ++round; }
+                    issued += ng;
+                    stage += ng;
+                    if (stage >= n_stages) { stage -= n_stages; ++round; }
+                    if (ng < kIssueGroup && ks + ng < nK) ks += ng - kIssueGroup;   // fewer stages than a group
                 }
             }
             if (s_abort && pid == 0) {
