@@ -37,11 +37,12 @@ constexpr int kMaxRows = 16384;
 
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-// Rows up to which the CUDA-core streaming kernel is taken.  Measured on the 3584 x 152064 head (us per call):
-//   rows       1      2      3      4      8
-//   streaming  160    175    211    228    453     (contiguous bulk copies: the best DRAM pattern, FMA-bound from 3 rows)
-//   tcgen05    173    179    176    178    184     (128-byte pieces of many rows per copy: ~7 % slower streaming)
-constexpr int kGemvMaxRows = 2;
+// Rows up to which the CUDA-core streaming kernel is taken.  Measured (us per call, rows 1 / 2 / 3 / 4 / 8):
+//   3584 x 152064 head   streaming 160 / 175-189 / 211 / 228 / 453    tcgen05 171 / 173 / 175 / 173 / 173
+//   1536 x 151936 head   streaming  77 /  79     / 100 / 101 / 186    tcgen05  81 /  81 /  81 /  82 /  82
+// One row streams best as contiguous bulk copies; from two rows on the FMA work shows (and more so on a
+// power-capped GPU), while the tensor-core kernel costs the same from 1 to 128 rows.
+constexpr int kGemvMaxRows = 1;
 
 size_t ws_partials_bytes(int R, int V)
 {

@@ -145,7 +145,7 @@ def test_tensor_core_path_nan_row_and_determinism(rs, handle, oracle):
 
 def test_path_choice(rs):
     assert rs.path_name(1, 1536, 151936) == "gemv" and rs.path_name(4, 3584, 152064) == "umma"
-    assert rs.path_name(2, 3584, 152064) == "gemv" and rs.path_name(3, 3584, 152064) == "umma"
+    assert rs.path_name(2, 3584, 152064) == "umma" and rs.path_name(3, 3584, 152064) == "umma"
     assert rs.path_name(16, 3584, 152064) == "umma" and rs.path_name(544, 5120, 152064) == "umma"
     assert rs.path_name(64, 32, 4096) == "gemv"          # too small for the tensor-core tiles
     assert rs.path_name(64, 1536, 151936, rs.PATH_GEMV) == "gemv"
