@@ -133,14 +133,14 @@ def measured_peaks() -> dict:
 # once any of them has changed the counters no longer describe the kernel and the figure reads null.
 NCU_TRAFFIC = {
     "c2_slm_b1":
-    {"bytes": 471142400, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
-     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "0f73425c4cb67810f1adb034f8e18534119ded82a547f9cf295d8c52e9fd561f", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 471505408, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
+     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
     "c4_slm_b64":
-    {"bytes": 471890176, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
-     "sources": {"rstitch_umma.cu": "44e4753e7db25c6c2bd1eb75550c6565b60f03e0f6112c88ce7063728df15ded", "rstitch_kernels.cuh": "0f73425c4cb67810f1adb034f8e18534119ded82a547f9cf295d8c52e9fd561f", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 471650048, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
+     "sources": {"rstitch_umma.cu": "81b3aa33b167d774c649775cee3a7f5f3977df1dc72a6144c72ccb9b47ba8d66", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
     "c5_catchup":
-    {"bytes": 1673879808, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
-     "sources": {"rstitch_umma.cu": "44e4753e7db25c6c2bd1eb75550c6565b60f03e0f6112c88ce7063728df15ded", "rstitch_kernels.cuh": "0f73425c4cb67810f1adb034f8e18534119ded82a547f9cf295d8c52e9fd561f", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "50a2ad89de04a8274efe6388b4182c37e5920ab689529df9fe702c85036f317a", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 1672147528, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
+     "sources": {"rstitch_umma.cu": "81b3aa33b167d774c649775cee3a7f5f3977df1dc72a6144c72ccb9b47ba8d66", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
 }
 
 
