@@ -3,22 +3,23 @@
 // tile into single-pass softmax statistics and the greedy token without the logits ever leaving
 // the SM.
 //
-// Block = 6 warps, one block per SM:
-//   warp 0  producer: one thread issues tensor-map (TMA) copies of a 128 x 64 hidden tile and an
-//           N x 64 W_head tile (128-byte swizzle) into a 4-stage shared-memory ring;
-//   warp 1  one thread issues the tcgen05.mma instructions (M = 128, N <= 256, K = 16) and commits
+// head_umma_kernel (at most 128 rows: one M tile).  Block = 10 warps, one block per SM:
+//   warp 0  producer: one thread issues tensor-map (TMA) copies of the hidden tile and an N x 64 W_head
+//           tile (128-byte swizzle) into a shared-memory ring of up to eight stages, two k-steps at a time;
+//   warp 1  one thread issues the tcgen05.mma instructions (M = 128 or 64, N <= 256, K = 16) and commits
 //           them to the ring's "empty" barriers and to the accumulator's "full" barrier; the warp
 //           also owns the tensor-memory allocation (512 columns = two 256-column accumulators);
-//   warps 2-5  epilogue: thread = one hidden row (one TMEM lane); it reads its row of the
-//           accumulator 32 columns at a time and folds the logits into (m, s, u, argmax).
+//   warps 2-9  epilogue: thread = one hidden row (one TMEM lane); it reads its row of the accumulator
+//           32 columns at a time and folds the logits into (m, s, u, argmax); warps 2-5 take the first
+//           half of a tile's columns, warps 6-9 the second.
 // The two accumulators alternate, so the epilogue of one tile runs under the MMAs of the next.
+// Each block owns one contiguous, balanced range of the vocabulary, cut into tiles of at most 256 rows,
+// and keeps one running statistic per row; W_head is read from HBM exactly once and the kernel is
+// HBM-bound.
 //
-// Work split.  Up to 128 rows (one M tile): each block owns one contiguous, balanced range of the
-// vocabulary, cut into tiles of at most 256 rows, and keeps one running statistic per row; W_head
-// is read from HBM exactly once and the kernel is HBM-bound.  More rows: work items are
-// (256-row vocabulary tile, 128-row M tile) pairs dealt round-robin with the M tiles of one
-// vocabulary tile adjacent, so that they run at the same time on neighbouring SMs and W_head
-// comes from HBM once and from L2 for the other M tiles.
+// head_umma2_kernel (more rows): work items are (256-row vocabulary tile, pair of 128-row M tiles) dealt
+// round-robin with the pairs of one vocabulary tile adjacent, so that they run at the same time on
+// neighbouring SMs and W_head comes from HBM once and from L2 for the others; see the comment there.
 #include "rstitch_kernels.cuh"
 #include "rstitch_ptx.cuh"
 
@@ -28,10 +29,11 @@ namespace rstitch {
 
 namespace {
 
-constexpr int kProducers = 1;                        // copy-issuing warps.  One thread issues ~7 tensor-map copies per
-                                                     // microsecond and separate warps issue in parallel (a probe reached
-                                                     // 19/us with four), but these kernels need at most ~6/us and measured
-                                                     // the same with 1, 2 and 3; the dealing code below stays general
+constexpr int kProducers = 1;                        // copy-issuing warps of the many-row kernels.  One thread issues ~7
+                                                     // tensor-map copies per microsecond and separate warps issue in
+                                                     // parallel (a probe reached 19/us with four), but these kernels need at
+                                                     // most ~6/us and measured the same with 1, 2 and 3; their dealing code
+                                                     // stays general
 // k-steps whose copies the one-M-tile kernel issues together.  Measured on the 3584 x 152064 head with 16
 // rows: 1 -> 197 us, 2 -> 181 us, 4 -> 200 us (a group needs that many free stages at once; with eight
 // stages a group of four leaves too little in flight).
