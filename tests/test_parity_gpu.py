@@ -487,3 +487,28 @@ def test_bounded_wait_runs_out_and_the_handle_stays_usable(rs, handle, oracle):
     for flags in (rs.PATH_GEMV, rs.PATH_UMMA):
         check_case(rs, handle, oracle, w, [0], flags=flags)          # asserts a clean status word again
     assert torch.cuda.is_available()
+
+
+def test_random_shapes_sweep(rs, handle, oracle):
+    # seeded draw of shapes across both kernel families: odd hidden sizes (k-steps that do not fill a group,
+    # half-empty last k-step), vocabularies that end inside a 16-row unit, row counts around the M-tile and
+    # M = 64 boundaries, last rounds that split into pieces
+    rng = np.random.default_rng(20260)
+    edges = [1, 2, 3, 8, 9, 16, 17, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 320, 385, 512, 640]
+    done = 0
+    while done < 48:
+        B = int(rng.choice(edges)) if rng.random() < 0.7 else int(rng.integers(1, 700))
+        d = 8 * int(rng.integers(1, 129))
+        V = int(rng.integers(2, 6000))
+        if B * d * V > 2.5e8:
+            continue
+        path = rng.choice(["auto", "gemv", "umma"])
+        if path == "gemv" and B > 40:
+            path = "auto"
+        flags = {"auto": 0, "gemv": rs.PATH_GEMV, "umma": rs.PATH_UMMA}[str(path)]
+        w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=d, V=V, seed=31000 + done, sigma_w=0.5 / math.sqrt(d))
+        try:
+            check_case(rs, handle, oracle, w, [0], flags=flags)
+        except AssertionError as e:
+            raise AssertionError("case %d: B=%d d=%d V=%d path=%s: %s" % (done, B, d, V, path, e))
+        done += 1
