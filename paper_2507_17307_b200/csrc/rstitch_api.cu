@@ -490,9 +490,25 @@ int rstitch_route_ex_host(rstitch_handle_t h, const rstitch_args_t *a, void *cud
             return n == 0 || cudaMemcpyAsync(base + o, src, n, cudaMemcpyHostToDevice, stream) == cudaSuccess;
         };
         ok = h2d(o_hid, a->hidden, n_src * a->d * 2);
-        if (ok && a->row_idx) ok = h2d(o_ridx, a->row_idx, R * 4);
-        if (ok && a->row_seq) ok = h2d(o_rseq, a->row_seq, R * 4);
-        if (ok && a->seq_len) ok = h2d(o_slen, a->seq_len, B * 4) && h2d(o_klen, a->kv_len, B * 4);
+        const size_t idx_bytes = o_tok - o_ridx;        // the index arrays follow the hidden rows
+        const bool any_idx = a->row_idx || a->row_seq || a->seq_len;
+        if (ok && any_idx && idx_bytes <= kPackedInputMax) {
+            // a large batch of rows: they go as they are, the small index arrays still as one copy
+            if (h->st_in_bytes < kPackedInputMax) {
+                if (h->st_in) { cudaFreeHost(h->st_in); h->st_in = nullptr; h->st_in_bytes = 0; }
+                if (cudaMallocHost(&h->st_in, kPackedInputMax) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
+                h->st_in_bytes = kPackedInputMax;
+            }
+            char *in = (char *)h->st_in - o_ridx;
+            if (a->row_idx) std::memcpy(in + o_ridx, a->row_idx, R * 4);
+            if (a->row_seq) std::memcpy(in + o_rseq, a->row_seq, R * 4);
+            if (a->seq_len) { std::memcpy(in + o_slen, a->seq_len, B * 4); std::memcpy(in + o_klen, a->kv_len, B * 4); }
+            ok = cudaMemcpyAsync(base + o_ridx, h->st_in, idx_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+        } else {
+            if (ok && a->row_idx) ok = h2d(o_ridx, a->row_idx, R * 4);
+            if (ok && a->row_seq) ok = h2d(o_rseq, a->row_seq, R * 4);
+            if (ok && a->seq_len) ok = h2d(o_slen, a->seq_len, B * 4) && h2d(o_klen, a->kv_len, B * 4);
+        }
     }
     if (!ok) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
 
