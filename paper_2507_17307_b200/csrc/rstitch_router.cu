@@ -6,7 +6,8 @@
 //     x0 = W_in s + b_in;  x <- x + W2_l GELU(W1_l x + b1_l) + b2_l;  y = LayerNorm(x) g + beta;
 //     logits = W_out y + b_out   (exact erf GELU, eps = 1e-5).
 // One block per row: the d -> h projection is spread over the block's warps (coalesced fp32 weight
-// rows against the bf16 hidden row held in shared memory), the small blocks run on one warp.
+// rows against the bf16 hidden row held in shared memory); narrow residual blocks, the normalisation and
+// the head run on one warp, wide blocks on all of them.
 #include "../../include/rstitch.h"
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -15,6 +16,7 @@ namespace {
 
 constexpr int kThreads = 512;
 constexpr int kMaxH = 256, kMaxFF = 1024;
+constexpr int kWarpStackMax = 8192;              // h * ff up to which one warp runs the residual blocks
 
 __device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
 {
@@ -42,6 +44,52 @@ __device__ __forceinline__ float warp_sum(float v)
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
+}
+
+// sum_k a[k] v[k] over k = 0 .. len-1, visited from element `start` on (mod len): the lanes of a warp,
+// each on a row of its own, then read 32 different banks whatever the row stride.  Four independent
+// chains; with a power-of-two length the indices need no wrap test and the loads run ahead of the FMAs.
+__device__ __forceinline__ float dot_rotated(const float *a, const float *v, int len, int start)
+{
+    float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
+    if (len >= 16 && (len & (len - 1)) == 0) {
+        // sixteen elements at a time, every load issued before the first FMA: a single warp has nothing
+        // else to hide the shared-memory latency with
+        const int m = len - 1;
+        for (int n = 0; n < len; n += 16) {
+            float av[16], vv[16];
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                const int k = (n + q + start) & m;
+                av[q] = a[k];
+                vv[q] = v[k];
+            }
+#pragma unroll
+            for (int q = 0; q < 16; q += 4) {
+                c0 = fmaf(av[q], vv[q], c0);
+                c1 = fmaf(av[q + 1], vv[q + 1], c1);
+                c2 = fmaf(av[q + 2], vv[q + 2], c2);
+                c3 = fmaf(av[q + 3], vv[q + 3], c3);
+            }
+        }
+    } else if (len >= 4 && (len & (len - 1)) == 0) {
+        const int m = len - 1;
+#pragma unroll 4
+        for (int n = 0; n < len; n += 4) {
+            const int k0 = (n + start) & m, k1 = (n + 1 + start) & m, k2 = (n + 2 + start) & m, k3 = (n + 3 + start) & m;
+            c0 = fmaf(a[k0], v[k0], c0);
+            c1 = fmaf(a[k1], v[k1], c1);
+            c2 = fmaf(a[k2], v[k2], c2);
+            c3 = fmaf(a[k3], v[k3], c3);
+        }
+    } else {
+        int k = start % len;
+        for (int n = 0; n < len; ++n) {
+            c0 = fmaf(a[k], v[k], c0);
+            if (++k == len) k = 0;
+        }
+    }
+    return (c0 + c1) + (c2 + c3);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -120,7 +168,24 @@ router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const
     }
     if (threadIdx.x < w.h) x[threadIdx.x] += p_b_in[threadIdx.x];
     __syncthreads();
-    for (int l = 0; l < w.n_blocks; ++l) {                          // residual FFN blocks
+    // Narrow blocks (the paper's router has ~0.17 M parameters, nearly all of them in W_in): with every
+    // weight already in shared memory one warp runs the whole stack, a lane per output, synchronising
+    // with __syncwarp only; sixteen warps sharing these tiny products spent ~3300 cycles per block on
+    // block-wide barriers and shuffle trees.
+    const bool warp_stack = stage_weights == 2 && w.h * w.ff <= kWarpStackMax;
+    if (warp_stack && warp != 0) return;
+    for (int l = 0; warp_stack && l < w.n_blocks; ++l) {
+        const float *w1 = blk + (size_t)l * per_block, *w2 = w1 + w.ff * w.h;
+        for (int j = lane; j < w.ff; j += 32) {
+            const float a = p_b1[(size_t)l * w.ff + j] + dot_rotated(w1 + (size_t)j * w.h, x, w.h, lane);
+            t[j] = 0.5f * a * (1.0f + erff(a * 0.70710678118654752f));      // exact GELU
+        }
+        __syncwarp();
+        for (int i = lane; i < w.h; i += 32)                                 // residual; x[i] has one reader here
+            x[i] += p_b2[(size_t)l * w.h + i] + dot_rotated(w2 + (size_t)i * w.ff, t, w.ff, lane);
+        __syncwarp();
+    }
+    for (int l = 0; !warp_stack && l < w.n_blocks; ++l) {           // residual FFN blocks, wide: the whole block
         const float *w1 = w.W1 + (size_t)l * w.ff * w.h, *w2 = w.W2 + (size_t)l * w.h * w.ff;
         if (stage_weights == 2) {
             w1 = blk + (size_t)l * per_block;
