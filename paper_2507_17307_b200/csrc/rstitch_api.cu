@@ -31,6 +31,7 @@ struct rstitch_handle_s {
 
 namespace {
 
+constexpr size_t kMirrorMax = 16 * 1024;        // host-buffer calls: outputs up to this size are written to the host by the kernel
 constexpr size_t kPackedInputMax = 64 * 1024;   // host-buffer calls: inputs up to this size travel as one copy
 constexpr int kMaxD = 16384;
 constexpr int kMaxRows = 16384;
@@ -220,8 +221,10 @@ bool make_alg1_tail(const rstitch_alg1_tail_t *t, Alg1Tail *out)
 
 // Validated arguments -> kernels.  With shard_stats the head is a vocabulary shard starting at entry
 // v_base: per-row statistics go to shard_stats and no routing output is touched.
+struct Mirror { const void *src = nullptr; void *dst = nullptr; size_t bytes = 0; };
+
 int enqueue_head(rstitch_handle_s *h, const rstitch_args_t *a, cudaStream_t stream, float *shard_stats,
-                        int v_base)
+                 int v_base, Mirror mirror = Mirror())
 {
     Alg1Tail alg1;
     if (!make_alg1_tail(shard_stats ? nullptr : a->alg1_tail, &alg1)) return RSTITCH_ERR_INVALID_ARG;
@@ -265,6 +268,8 @@ int enqueue_head(rstitch_handle_s *h, const rstitch_args_t *a, cudaStream_t stre
     ta.stat = h->stat;
     ta.shard_stats = shard_stats; ta.v_base = v_base;
     ta.alg1 = alg1;
+    ta.mirror_src = (const uint4 *)mirror.src; ta.mirror_dst = (uint4 *)mirror.dst;
+    ta.mirror_vec = (uint32_t)(mirror.bytes / 16);
 
     void *ws = a->workspace ? a->workspace : h->ws;
     Scratch sc = scratch_carve(ws);
@@ -402,6 +407,7 @@ int rstitch_shard_route(rstitch_handle_t h, const rstitch_args_t *a, const void 
     ta.stat = h->stat;
     ta.shard_stats = nullptr; ta.v_base = 0;
     ta.alg1 = alg1;
+    ta.mirror_src = nullptr; ta.mirror_dst = nullptr; ta.mirror_vec = 0;
     Scratch sc = scratch_carve(h->ws);
     int launched = 0;
     cudaError_t e = launch_shard_merge((const float *)gathered, n_shards, a->n_rows_dev, ta, sc.ticket, stream,
@@ -526,18 +532,31 @@ int rstitch_route_ex_host(rstitch_handle_t h, const rstitch_args_t *a, void *cud
     dv.llm_row_off = a->seq_len ? (int32_t *)(base + o_roff) : nullptr;
     dv.llm_count = (int32_t *)(base + o_cnt);
     dv.route_mask = (uint8_t *)(base + o_msk);
-    st = rstitch_route_ex(h, &dv, cuda_stream);
-    if (st != RSTITCH_OK) return st;
-
-    // the outputs are contiguous in the staging block: one copy into a pinned mirror, then plain
-    // host copies into the caller's buffers (a handful of small device-to-host copies costs more)
+    // The outputs are contiguous in the staging block and go to a pinned mirror in one piece, then with
+    // plain host copies into the caller's buffers (a handful of small device-to-host copies costs more).
+    // A few KB are written there by the deciding block itself (the mirror is mapped into the device's
+    // address space), which saves the copy command and its latency; more goes through a copy.
     const size_t out_bytes = off - o_tok;
     if (out_bytes > h->st_host_bytes) {
         if (h->st_host) { cudaFreeHost(h->st_host); h->st_host = nullptr; h->st_host_bytes = 0; }
         if (cudaMallocHost(&h->st_host, out_bytes) != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
         h->st_host_bytes = out_bytes;
     }
-    ok = cudaMemcpyAsync(h->st_host, base + o_tok, out_bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+    Mirror mirror;
+    void *mirror_dev = nullptr;
+    if (out_bytes <= kMirrorMax && dv.alg1_tail == nullptr &&
+        cudaHostGetDevicePointer(&mirror_dev, h->st_host, 0) == cudaSuccess && mirror_dev) {
+        mirror.src = base + o_tok; mirror.dst = mirror_dev; mirror.bytes = out_bytes;
+    } else {
+        cudaGetLastError();
+    }
+    st = validate(h, &dv);
+    if (st != RSTITCH_OK) return st;
+    h->last_stream = stream;
+    st = enqueue_head(h, &dv, stream, nullptr, 0, mirror);
+    if (st != RSTITCH_OK) return st;
+    ok = (mirror.dst != nullptr ||
+          cudaMemcpyAsync(h->st_host, base + o_tok, out_bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess) &&
          cudaStreamSynchronize(stream) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
     const char *hb = (const char *)h->st_host - o_tok;

@@ -93,6 +93,7 @@ extern "C" int rstitch_route_static(const void *hidden, const void *W_head, int 
     ta.stat = (DevStat *)((char *)base + kStatOffset);
     ta.shard_stats = nullptr; ta.v_base = 0;
     ta.alg1.on = 0;
+    ta.mirror_src = nullptr; ta.mirror_dst = nullptr; ta.mirror_vec = 0;
     Scratch sc = scratch_carve(base);
     cudaError_t e = launch_head_gemv(ha, ta, sc, sms, stream);
     if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }

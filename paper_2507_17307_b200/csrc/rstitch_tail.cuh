@@ -70,6 +70,12 @@ struct TailArgs {
     float   *shard_stats;        // [R][5] or nullptr
     int      v_base;
     Alg1Tail alg1;               // optional: Algorithm 1's decision block (and the next round's plans) after S6
+    // Host-buffer calls: after everything else the deciding block copies the call's outputs (one contiguous
+    // piece of device memory, a multiple of 16 bytes) to pinned host memory mapped into the device's address
+    // space, which saves the device-to-host copy command and its latency.  nullptr: no copy.
+    const uint4 *mirror_src;
+    uint4       *mirror_dst;
+    uint32_t     mirror_vec;     // number of 16-byte words
 };
 
 constexpr int kShardWords = 5;
@@ -403,6 +409,10 @@ __device__ inline void tail_route(const TailArgs &a, int *smem)
                      a.llm_row_off, a.stat, smem);
     }
     if (a.alg1.on) alg1_tail_block(a.alg1, a.tok_out, a.route_mask, smem);
+    if (a.mirror_dst) {
+        __syncthreads();             // the block's own output stores; other blocks' came before the ticket
+        for (uint32_t i = threadIdx.x; i < a.mirror_vec; i += blockDim.x) a.mirror_dst[i] = __ldcg(a.mirror_src + i);
+    }
 }
 
 }  // namespace rstitch
