@@ -133,14 +133,14 @@ def measured_peaks() -> dict:
 # once any of them has changed the counters no longer describe the kernel and the figure reads null.
 NCU_TRAFFIC = {
     "c2_slm_b1":
-    {"bytes": 471505408, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
-     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 471337088, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
+     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "cd4da5f27447a88d28393e5aa40a8d6bdecfbe7ab8da0e06d678a01268d9b48f", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
     "c4_slm_b64":
-    {"bytes": 471650048, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
-     "sources": {"rstitch_umma.cu": "b0f379310c237b685275d916050df3d5b03d32f0860c865a399007a73dba3a39", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 472086784, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
+     "sources": {"rstitch_umma.cu": "b0f379310c237b685275d916050df3d5b03d32f0860c865a399007a73dba3a39", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "cd4da5f27447a88d28393e5aa40a8d6bdecfbe7ab8da0e06d678a01268d9b48f", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
     "c5_catchup":
-    {"bytes": 1672147528, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
-     "sources": {"rstitch_umma.cu": "b0f379310c237b685275d916050df3d5b03d32f0860c865a399007a73dba3a39", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "e1acfa507316cbf0684b0b01f07daf7489b5ca42fb7f8010e01ad48fab211589", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 1667069088, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
+     "sources": {"rstitch_umma.cu": "b0f379310c237b685275d916050df3d5b03d32f0860c865a399007a73dba3a39", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "cd4da5f27447a88d28393e5aa40a8d6bdecfbe7ab8da0e06d678a01268d9b48f", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
 }
 
 
