@@ -229,3 +229,88 @@ def test_argument_errors(rs):
     assert L.rstitch_alg1_init(None, 4, None, None) == -1
     assert L.rstitch_alg1_commit(C.byref(st._c), 4, 0, None, None, None, None, None, 0, None) == -1
     torch.cuda.synchronize()
+
+
+def test_fused_loop_replays_from_one_cuda_graph(rs, oracle):
+    # several rounds of the hybrid loop -- two routing calls per round, Algorithm 1's decision block and the
+    # planning inside them, nothing on the host -- recorded into ONE CUDA graph; replaying it gives the state
+    # the same calls give when issued directly, and that state matches the oracle's per-sequence loop
+    import torch
+    # T_max = the number of rounds: the planning the last LLM call carries then selects nothing, so the state
+    # is the one Algorithm 1 leaves after T_max iterations
+    B, rounds, tau, eos = 48, 6, 0.3, -1
+    c = coeffs()
+    lat = [rs.LatencyModel(*c["SLM-1.5B"]), rs.LatencyModel(*c["LLM-7B"])]
+    for seed in range(20):
+        ws = [gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=256, V=2053, seed=8400 + seed, diffuse_frac=(0.4, 0.4)),
+              gen.scaled(gen.WORKLOADS["c4_llm_b64"], B=B, d=320, V=3001, seed=8500 + seed, diffuse_frac=(0.6, 0.6))]
+        w_bits = [gen.make_w_head(w) for w in ws]
+        # run entry j of a model's batch reads row j of that model's pool in every round
+        pools_bits = [gen.make_hidden(ws[m], w_bits[m], 0)[0] for m in (0, 1)]
+        refs = [oracle.route(pools_bits[m], w_bits[m], tau) for m in (0, 1)]
+        if all((np.abs(r["ent"] - tau) > 4 * ENT_TOL).all() and (r["gap"] > GAP_TOL).all() for r in refs):
+            break
+    else:
+        raise AssertionError("no seed kept every row clear of the tolerance bands")
+    w_dev = [to_dev_bf16(b) for b in w_bits]
+    pools = [to_dev_bf16(p) for p in pools_bits]
+    prompt = to_dev_i32(np.arange(3, 3 + B))
+    handles = [rs.Handle(64, 256, 4096), rs.Handle(64, 320, 4096)]
+    side = torch.cuda.Stream()
+
+    def make(state):
+        tails = [state.tail(0, eos, spans=False), state.tail(1, eos, spans=False, plan_next=True, t_max=rounds, latency=lat)]
+        outs = [rs.RouteOutputs.allocate(B, B, "cuda") for _ in (0, 1)]
+        calls = [rs.PreparedCall(handles[m], pools[m], w_dev[m], tau, outs[m], n_rows_dev=state.run_count[m],
+                                 stream=side, alg1_tail=tails[m]) for m in (0, 1)]
+        return calls, tails, outs
+
+    def start(state):
+        with torch.cuda.stream(side):
+            state.init(prompt, stream=side)
+            state.plan(0, rounds, lat[0], stream=side)
+            state.plan(1, rounds, lat[1], stream=side)
+
+    direct, graphed = rs.Alg1State(B, y_cap=rounds), rs.Alg1State(B, y_cap=rounds)
+    calls_d, keep_d, _ = make(direct)
+    start(direct)
+    with torch.cuda.stream(side):
+        for _ in range(rounds):
+            assert calls_d[0].launch() == 0 and calls_d[1].launch() == 0
+    side.synchronize()
+
+    calls_g, keep_g, _ = make(graphed)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        for _ in range(rounds):
+            assert calls_g[0].launch() == 0 and calls_g[1].launch() == 0
+    start(graphed)            # the capture ran nothing: the state starts here
+    side.synchronize()
+    g.replay()
+    torch.cuda.synchronize()
+    a, b = state_to_host(direct), state_to_host(graphed)
+    for k in a:
+        assert np.array_equal(a[k], b[k]), k
+    assert a["kept"][1].sum() > 0 and a["kept"][0].sum() > 0        # both models produced tokens
+    # against the oracle: sequence b saw (token, entropy) of pool row j whenever it was run entry j; with
+    # every sequence alive in every round the run lists are the ascending ids of each model's sequences,
+    # which the oracle's own loop reproduces when fed the per-round streams recorded below
+    active = np.zeros(B, dtype=np.int64)
+    tok_s = np.zeros((2, B, rounds), dtype=np.int32)
+    ent_s = np.zeros((2, B, rounds))
+    for t in range(rounds):
+        nxt = active.copy()
+        for m in (0, 1):
+            ids = np.flatnonzero(active == m)
+            for j, sid in enumerate(ids):
+                tok_s[m, sid, t], ent_s[m, sid, t] = refs[m]["tok"][j], refs[m]["ent"][j]
+                routed = refs[m]["ent"][j] > tau
+                nxt[sid] = 1 if (m == 0 and routed) or (m == 1 and routed) else 0
+        active = nxt
+    for sid in range(B):
+        ref = oracle.alg1_sequence(3 + sid, rounds, tau, eos, tok_s[0, sid], ent_s[0, sid], tok_s[1, sid], ent_s[1, sid],
+                                   c["SLM-1.5B"], c["LLM-7B"])
+        check_against_oracle(oracle, a, sid, ref)
+    for h in handles:
+        assert rs.last_status(h)["timeouts"] == 0
+        h.destroy()
