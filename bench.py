@@ -658,6 +658,9 @@ def main() -> int:
                        "cuda_graph": bool(args.graph)},
             "roofline": roof, "clocks": clocks.summary(), "gpu_launches": launches,
             "algorithmic_bytes_per_step": algo_bytes, "flops_per_step": flops,
+            # `value` counts rows (every row gets a token and an entropy); with multi-row spans a sequence
+            # is decided by its last row, so the sequences decided per second are fewer
+            "rows_per_s": value, "sequences_per_s": world * w0.B * K / sec,
         }
         line["e2e"] = {"value": world * decisions_per_step * e2e["steps"] / e2e["seconds"], "unit": UNIT,
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
