@@ -43,8 +43,8 @@ BENCH_WORKLOADS = {
     # launches: the SLM head on the sequences decoding on the SLM, the LLM head on the others, each applying
     # Algorithm 1's decision block in its own tail, the LLM's call also planning the next round
     "alg1_b64": ("c4_slm_b64", "c4_llm_b64"),
-    # R-Stitch+ step: SLM head on 64 sequences, the router on the rows the entropy rule routed, compaction
-    # of the router's refined mask
+    # R-Stitch+ step, two launches: SLM head on 64 sequences, then the router on the rows the entropy rule
+    # routed with the compaction of its refined mask in the same kernel
     "c4_router": ("c4_slm_b64",),
 }
 
@@ -481,15 +481,14 @@ def main() -> int:
                 raise rs.RstitchError(st, "rstitch_route_ex")
         if with_router:
             o = calls[0].out
-            router.forward(calls[0]._keep[1], 64, row_idx=o.llm_idx, n_rows_dev=o.llm_count, logits=r_logits,
-                           switch=r_switch, refine_mask=o.mask, stream=stream)
-            rs.compact(o.mask, r_idx, r_cnt, stream=stream)
+            router.route(calls[0]._keep[1], 64, o.llm_idx, o.mask, r_idx, r_cnt, n_rows_dev=o.llm_count,
+                         logits=r_logits, switch=r_switch, stream=stream)
 
     for i in range(Wm):
         step(i)
     torch.cuda.synchronize()
     warm_launches = sum(rs.last_status(hd)["launches"] for hd in handles)     # also clears the counters
-    launches_per_step = warm_launches / float(Wm) + (2 if with_router else 0)
+    launches_per_step = warm_launches / float(Wm) + (1 if with_router else 0)
 
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if dist is not None:
@@ -535,7 +534,7 @@ def main() -> int:
         dist.barrier()
     ms = ev0.elapsed_time(ev1)
     stats = [rs.last_status(hd) for hd in handles]
-    launches = sum(st["launches"] for st in stats) + (2 * K if with_router else 0)
+    launches = sum(st["launches"] for st in stats) + (1 * K if with_router else 0)
     if graph is not None:
         launches = int(round(K * launches_per_step))      # replayed kernels are not counted by the handles
     if any(st["timeouts"] or st["nan_rows"] for st in stats):

@@ -317,6 +317,19 @@ int rstitch_router_forward(const rstitch_router_t *w, const void *hidden, int n_
                            const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out,
                            uint8_t *refine_mask, void *cuda_stream);
 
+/*
+ * The R-Stitch+ decision in one launch: rstitch_router_forward with refine_mask = route_mask, followed in
+ * the same kernel (its last block to finish) by the ordered compaction of the refined route_mask [n_src]
+ * into llm_idx [n_src] and llm_count [1], exactly as rstitch_compact(route_mask, n_src, ...) would give
+ * afterwards.  row_idx, route_mask and llm_count are required; typically row_idx = llm_idx of the SLM head's
+ * call (the list is consumed before it is rewritten only if the two are DIFFERENT buffers: pass another
+ * llm_idx here).  n_src <= 65536.  Calls of this function that may overlap on one device must be ordered
+ * by the caller (they share one ticket counter).
+ */
+int rstitch_router_route(const rstitch_router_t *w, const void *hidden, int n_src, const int32_t *row_idx,
+                         const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out,
+                         uint8_t *route_mask, int32_t *llm_idx, int32_t *llm_count, void *cuda_stream);
+
 /* Handle: owns the scratch memory and the device status word for problems up to the given maxima on
  * the current device.  rstitch_destroy(NULL) is a no-op. */
 int rstitch_create(rstitch_handle_t *out, int maxR, int max_d, int maxV);

@@ -133,6 +133,8 @@ def lib():
         L.rstitch_shard_route.restype = i
         L.rstitch_router_forward.argtypes = [C.POINTER(_Router), vp, i, vp, vp, i, vp, vp, vp, vp]
         L.rstitch_router_forward.restype = i
+        L.rstitch_router_route.argtypes = [C.POINTER(_Router), vp, i, vp, vp, i, vp, vp, vp, vp, vp, vp]
+        L.rstitch_router_route.restype = i
         L.rstitch_alg1_init.argtypes = [C.POINTER(_Alg1State), i, vp, vp]
         L.rstitch_alg1_init.restype = i
         L.rstitch_alg1_plan.argtypes = [C.POINTER(_Alg1State), i, i, i, C.POINTER(LatencyModel), vp, vp, vp, vp, vp, vp]
@@ -580,4 +582,22 @@ class Router:
             return st
         if st != 0:
             raise RstitchError(st, "rstitch_router_forward")
+        return logits, switch
+
+    def route(self, hidden, R: int, row_idx, route_mask, llm_idx, llm_count, n_rows_dev=None, logits=None,
+              switch=None, stream=None, check: bool = True):
+        """rstitch_router_route: the router on the rows row_idx names, route_mask refined in place and
+        compacted into llm_idx / llm_count by the same launch; returns (logits, switch)."""
+        import torch
+        if logits is None:
+            logits = torch.zeros((max(R, 1), 2), dtype=torch.float32, device=hidden.device)
+        if switch is None:
+            switch = torch.full((max(R, 1),), 255, dtype=torch.uint8, device=hidden.device)
+        st = lib().rstitch_router_route(C.byref(self._c), _ptr(hidden), int(hidden.shape[0]), _ptr(row_idx),
+                                        _ptr(n_rows_dev), int(R), _ptr(logits), _ptr(switch), _ptr(route_mask),
+                                        _ptr(llm_idx), _ptr(llm_count), _stream_ptr(stream))
+        if not check:
+            return st
+        if st != 0:
+            raise RstitchError(st, "rstitch_router_route")
         return logits, switch

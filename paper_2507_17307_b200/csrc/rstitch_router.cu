@@ -8,8 +8,7 @@
 // One block per row: the d -> h projection is spread over the block's warps (coalesced fp32 weight
 // rows against the bf16 hidden row held in shared memory); narrow residual blocks, the normalisation and
 // the head run on one warp, wide blocks on all of them.
-#include "../../include/rstitch.h"
-#include <cuda_runtime.h>
+#include "rstitch_kernels.cuh"
 #include <math_constants.h>
 
 namespace {
@@ -112,17 +111,12 @@ __device__ __forceinline__ float dot_rotated4(const float4 *a, const float4 *v, 
     return (c0 + c1) + (c2 + c3);
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
-router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const int32_t *row_idx,
-              const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out, uint8_t *refine_mask,
-              int stage_weights)
+// One row by one block (every thread calls; warps other than the first may leave before the end).
+__device__ __forceinline__ void router_row(const rstitch_router_t &w, const unsigned short *hidden, int n_src,
+                                           const int32_t *row_idx, int r, float *logits_out, uint8_t *switch_out,
+                                           uint8_t *refine_mask, int stage_weights, float *sm)
 {
-    extern __shared__ __align__(16) float sm[];   // [d] hidden row | [h] x | [ff] t | [ff h] W1 | [h ff] W2 of a block
     float *s = sm, *x = sm + w.d, *t = x + w.h;
-    int R_live = R;
-    if (n_rows_dev) { int n = *n_rows_dev; R_live = n < 0 ? 0 : (n < R ? n : R); }
-    const int r = blockIdx.x;
-    if (r >= R_live) return;
     int src = row_idx ? row_idx[r] : r;
     if (src < 0 || src >= n_src) src = 0;
     const unsigned short *hrow = hidden + (size_t)src * w.d;
@@ -294,12 +288,40 @@ router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const
     }
 }
 
+// Ticket of the compacting form: the blocks of one launch count themselves here, the last one resets it.
+__device__ unsigned g_router_ticket = 0;
+
+// cmp_count == nullptr: the router alone.  Otherwise every block takes a ticket when its row is done and
+// the last one compacts refine_mask [n_src] into cmp_idx / cmp_count, as rstitch_compact would.
+__global__ void __launch_bounds__(kThreads, 1)
+router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const int32_t *row_idx,
+              const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out, uint8_t *refine_mask,
+              int stage_weights, int32_t *cmp_idx, int32_t *cmp_count)
+{
+    extern __shared__ __align__(16) float sm[];   // [d] hidden row | [h] x | [ff] t | [ff h] W1 | [h ff] W2 of a block
+    __shared__ int s_tail[66];
+    __shared__ int s_last;
+    int R_live = R;
+    if (n_rows_dev) { int n = *n_rows_dev; R_live = n < 0 ? 0 : (n < R ? n : R); }
+    const int r = blockIdx.x;
+    if (r < R_live) router_row(w, hidden, n_src, row_idx, r, logits_out, switch_out, refine_mask, stage_weights, sm);
+    if (cmp_count == nullptr) return;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(&g_router_ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    rstitch::tail_compact(refine_mask, n_src, nullptr, nullptr, cmp_idx, cmp_count, nullptr, nullptr, nullptr, s_tail);
+    if (threadIdx.x == 0) g_router_ticket = 0u;
+}
+
 }  // namespace
 
-extern "C" int rstitch_router_forward(const rstitch_router_t *w, const void *hidden, int n_src,
-                                      const int32_t *row_idx, const int32_t *n_rows_dev, int R,
-                                      float *logits_out, uint8_t *switch_out, uint8_t *refine_mask,
-                                      void *cuda_stream)
+static int router_launch(const rstitch_router_t *w, const void *hidden, int n_src,
+                         const int32_t *row_idx, const int32_t *n_rows_dev, int R,
+                         float *logits_out, uint8_t *switch_out, uint8_t *refine_mask,
+                         int32_t *cmp_idx, int32_t *cmp_count, void *cuda_stream)
 {
     if (!w || R < 0 || n_src < 0 || !logits_out) return RSTITCH_ERR_INVALID_ARG;
     if (w->d < 1 || w->h < 1 || w->ff < 1 || w->n_blocks < 0) return RSTITCH_ERR_INVALID_ARG;
@@ -335,7 +357,28 @@ extern "C" int rstitch_router_forward(const rstitch_router_t *w, const void *hid
     }
     router_kernel<<<R, kThreads, smem, (cudaStream_t)cuda_stream>>>(*w, (const unsigned short *)hidden, n_src, row_idx,
                                                                     n_rows_dev, R, logits_out, switch_out, refine_mask,
-                                                                    stage_weights);
+                                                                    stage_weights, cmp_idx, cmp_count);
     if (cudaGetLastError() != cudaSuccess) return RSTITCH_ERR_CUDA;
     return RSTITCH_OK;
+}
+
+extern "C" int rstitch_router_forward(const rstitch_router_t *w, const void *hidden, int n_src,
+                                      const int32_t *row_idx, const int32_t *n_rows_dev, int R,
+                                      float *logits_out, uint8_t *switch_out, uint8_t *refine_mask,
+                                      void *cuda_stream)
+{
+    return router_launch(w, hidden, n_src, row_idx, n_rows_dev, R, logits_out, switch_out, refine_mask, nullptr,
+                         nullptr, cuda_stream);
+}
+
+extern "C" int rstitch_router_route(const rstitch_router_t *w, const void *hidden, int n_src,
+                                    const int32_t *row_idx, const int32_t *n_rows_dev, int R,
+                                    float *logits_out, uint8_t *switch_out, uint8_t *route_mask,
+                                    int32_t *llm_idx, int32_t *llm_count, void *cuda_stream)
+{
+    if (!row_idx || !route_mask || !llm_count || (n_src > 0 && !llm_idx)) return RSTITCH_ERR_INVALID_ARG;
+    if (n_src > 65536) return RSTITCH_ERR_UNSUPPORTED_SHAPE;             // one block compacts the mask
+    if (R == 0) return rstitch_compact(route_mask, n_src, llm_idx, llm_count, cuda_stream);
+    return router_launch(w, hidden, n_src, row_idx, n_rows_dev, R, logits_out, switch_out, route_mask, llm_idx,
+                         llm_count, cuda_stream);
 }

@@ -77,6 +77,23 @@ def test_router_after_the_entropy_rule(rs, oracle):
     want_idx = np.flatnonzero(want_mask)
     assert int(cnt2.item()) == want_idx.size and np.array_equal(idx2.cpu().numpy()[:want_idx.size], want_idx)
     assert 0 < want_idx.size < cnt                        # the router kept some steps on the SLM
+    # the one-launch form: same refined mask, same compaction, three times in a row (the ticket rewinds)
+    for _ in range(3):
+        mask3 = out.mask.clone()
+        idx3 = torch.full((64,), -1, dtype=torch.int32, device="cuda")
+        cnt3 = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        logits3, sw3 = router.route(hid_dev, 64, out.llm_idx, mask3, idx3, cnt3, n_rows_dev=out.llm_count)
+        torch.cuda.synchronize()
+        assert torch.equal(mask3, mask) and torch.equal(logits3[:cnt], logits[:cnt]) and torch.equal(sw3, sw)
+        assert int(cnt3.item()) == want_idx.size and np.array_equal(idx3.cpu().numpy()[:want_idx.size], want_idx)
+        assert (idx3.cpu().numpy()[want_idx.size:] == -1).all()
+    # nothing routed by the entropy rule: the router has no rows, the compaction still runs
+    zero = torch.zeros(1, dtype=torch.int32, device="cuda")
+    mask0 = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    router.route(hid_dev, 64, out.llm_idx, mask0, idx3, cnt3, n_rows_dev=zero)
+    torch.cuda.synchronize()
+    assert int(cnt3.item()) == 0 and int(mask0.sum().item()) == 0
+    assert router.route(hid_dev, 64, None, mask0, idx3, cnt3, check=False) == -1       # row_idx is required
     handle.destroy()
 
 
