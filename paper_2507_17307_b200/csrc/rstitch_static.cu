@@ -3,9 +3,8 @@
 // Some users of this library run where cudaMalloc is off limits: inside a serving engine that has
 // handed all device memory to its own pool, in a latency-critical decode loop where an allocation
 // would synchronise the device, or in a process whose memory budget is fixed at start-up.  For
-// them the scratch of the split-V head kernel (the ticket counter, the per-slice partial
-// statistics and the status word) lives in a fixed array inside the library image instead of in a
-// handle.  Every GPU that loads the library holds that array until the process exits.
+// them the scratch of the head kernels (the ticket counter, the per-slice partial statistics and
+// the status word) lives in a fixed array inside the library image instead of in a handle.  Every GPU that loads the library holds that array until the process exits.
 #include "../../include/rstitch.h"
 #include "rstitch_kernels.cuh"
 
@@ -95,7 +94,17 @@ extern "C" int rstitch_route_static(const void *hidden, const void *W_head, int 
     ta.alg1.on = 0;
     ta.mirror_src = nullptr; ta.mirror_dst = nullptr; ta.mirror_vec = 0;
     Scratch sc = scratch_carve(base);
-    cudaError_t e = launch_head_gemv(ha, ta, sc, sms, stream);
+    // Same choice of kernel as the regular entry points: one row streams on the CUDA cores, more rows go
+    // to the tensor-core kernel (its tensor maps are encoded on the host and travel as kernel
+    // parameters, its accumulators live in tensor memory: no device allocation either; at most
+    // kStaticMaxRows x #blocks partials, well inside the array).
+    cudaError_t e;
+    if (B > 1 && umma_shape_ok(B, d, V)) {
+        int launched = 0;
+        e = launch_head_umma(ha, ta, sc, nullptr, sms, stream, &launched, false);
+    } else {
+        e = launch_head_gemv(ha, ta, sc, sms, stream);
+    }
     if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }
     return RSTITCH_OK;
 }
