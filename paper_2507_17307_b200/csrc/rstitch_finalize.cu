@@ -1,0 +1,90 @@
+// Cross-block finalisation of the head kernels as a launch of its own (S2-S6): one warp per row merges
+// the row's per-slice statistics in a fixed order and writes entropy and token; the last block to
+// finish applies the rule of Eq. 2, compacts and (optionally) carries Algorithm 1 on.
+//
+// The kernel is launched with programmatic stream serialisation behind the head kernel, and so is the
+// next call's head kernel behind this one.  A head kernel streams W_head -- a weight, which no kernel
+// of this library writes -- from its first instruction and only waits for the kernels before it when
+// it first needs something they may have written (hidden rows, index lists, the scratch).  Back to back,
+// step i + 1 therefore streams while step i's statistics are merged here, on a few warps that share an
+// SM with a streaming block, and no SM idles through the merge, the drain of the grid and the next launch.
+#include "rstitch_kernels.cuh"
+#include "rstitch_ptx.cuh"
+
+namespace rstitch {
+
+namespace {
+
+constexpr int kFinThreads = 128;
+constexpr int kFinRows    = kFinThreads / 32;        // one warp per row
+
+__global__ void __launch_bounds__(kFinThreads)
+head_finalize_kernel(Partials P, int n_slices, int R, const int32_t *n_rows_dev, TailArgs t, unsigned *ticket)
+{
+    __shared__ int s_tail[66];
+    __shared__ int s_last;
+    ptx::grid_dep_launch_dependents();
+    ptx::grid_dep_wait();                            // the head kernel has completed: its partials are visible
+    int R_live = R;
+    if (n_rows_dev) { int n = *n_rows_dev; R_live = n < 0 ? 0 : (n < R ? n : R); }
+    const int lane = threadIdx.x & 31;
+    for (int r = blockIdx.x * kFinRows + (threadIdx.x >> 5); r < R_live; r += gridDim.x * kFinRows) {
+        Stats st;
+        if (n_slices <= 256) {
+            st = tail_row_direct(P, (size_t)r * n_slices, n_slices, lane);
+        } else {
+            st = tail_merge_strided(P, (size_t)r * n_slices, n_slices, lane, 32);
+            stats_warp_allmerge(st);
+        }
+        if (lane == 0) tail_emit_row(st, r, t);
+    }
+    if (gridDim.x > 1) {
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned k = atomicAdd(ticket, 1u);
+            s_last = (k == gridDim.x - 1);
+        }
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+    } else {
+        __syncthreads();
+    }
+    TailArgs ta = t;
+    ta.R = R_live;
+    if (n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
+    tail_route(ta, s_tail);
+    if (gridDim.x > 1 && threadIdx.x == 0) *ticket = 0u;
+}
+
+}  // namespace
+
+cudaError_t launch_dependent(const void *func, dim3 grid, dim3 block, size_t smem, cudaStream_t stream, void **args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelExC(&cfg, func, args);
+}
+
+cudaError_t launch_head_finalize(const Partials &P, int n_slices, int R, const int32_t *n_rows_dev,
+                                 const TailArgs &t, unsigned *ticket, int sm_count, cudaStream_t stream)
+{
+    int grid = (R + kFinRows - 1) / kFinRows;
+    if (grid > sm_count) grid = sm_count;
+    if (grid < 1) grid = 1;
+    Partials p = P;
+    TailArgs ta = t;
+    void *args[] = {&p, &n_slices, &R, &n_rows_dev, &ta, &ticket};
+    return launch_dependent((const void *)head_finalize_kernel, dim3((unsigned)grid), dim3(kFinThreads), 0, stream, args);
+}
+
+}  // namespace rstitch

@@ -44,8 +44,11 @@ __device__ __forceinline__ void raise_abort(volatile int *flag, DevStat *stat, u
 // RT hidden rows per pass, VR vocabulary rows per ring slot.
 template <int RT, int VR>
 __global__ void __launch_bounds__(kThreads, 1)
-head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_slots, int hid_bytes)
+head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_slots, int hid_bytes, int split_tail)
 {
+    // split_tail: the merge of the slices and the routing tail run in head_finalize_kernel, launched
+    // behind this kernel; the next call's kernel may start as soon as this one's blocks leave their SMs.
+    if (split_tail) ptx::grid_dep_launch_dependents();
     extern __shared__ __align__(128) unsigned char dyn_smem[];   // [hidden RT x d][ring]
     __shared__ __align__(8) uint64_t s_full[kMaxSlots];
     __shared__ __align__(8) uint64_t s_empty[kMaxSlots];
@@ -64,7 +67,10 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
     const uint32_t row_bytes = (uint32_t)h.d * 2u;
     const uint32_t chunk_bytes = row_bytes * VR;
     int R_live = h.R;
-    if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
+    // A live row count on the device comes from the kernel before this one: wait for it.  Otherwise the
+    // producer streams W_head (which no earlier kernel writes) at once, and only the consumers wait,
+    // before they read the hidden rows.
+    if (h.n_rows_dev) { ptx::grid_dep_wait(); int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
     const int n_src = h.n_src > 0 ? h.n_src : h.R;
     const uint4 *H4 = (const uint4 *)h.hidden;
     uint4 *hid4 = (uint4 *)dyn_smem;
@@ -91,6 +97,7 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
         __syncthreads();                       // barriers ready: the producer may start at once
         // hidden rows of this pass -> shared memory (rows past the live count read as zero); only
         // the consumer warps take part, the producer is already streaming W_head
+        if (warp < kConsumerWarps) ptx::grid_dep_wait();      // earlier kernels' writes (hidden rows, scratch) are visible
         if (warp < kConsumerWarps)
         for (int i = threadIdx.x; i < RT * d8; i += kConsumerWarps * 32) {
             int r = r0 + i / d8, c = i - (i / d8) * d8;
@@ -205,6 +212,7 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
             ptx::mbar_wait(ptx::smem_u32(&s_full[j % n_slots]), (uint32_t)((j / n_slots) & 1), &s_zero);
     }
 
+    if (split_tail) return;                    // head_finalize_kernel merges the slices and decides
     // last block done: merge all slices and run the routing tail
     __threadfence();
     __syncthreads();
@@ -249,7 +257,7 @@ Plan make_plan(int R, int d)
 
 template <int RT, int VR>
 cudaError_t launch_inst(const HeadArgs &h, const TailArgs &t, const Scratch &s, const Plan &p, int grid,
-                        cudaStream_t stream)
+                        cudaStream_t stream, bool split_tail, int sm_count)
 {
     static bool configured[64] = {};
     int dev = 0;
@@ -262,28 +270,38 @@ cudaError_t launch_inst(const HeadArgs &h, const TailArgs &t, const Scratch &s, 
         configured[dev] = true;
     }
     Partials P = partials_carve(s.partials, (size_t)h.R, (size_t)grid);
-    head_stream_kernel<RT, VR><<<grid, kThreads, p.smem, stream>>>(h, t, P, s.ticket, p.n_slots, p.hid_bytes);
-    return cudaGetLastError();
+    if (!split_tail) {
+        head_stream_kernel<RT, VR><<<grid, kThreads, p.smem, stream>>>(h, t, P, s.ticket, p.n_slots, p.hid_bytes, 0);
+        return cudaGetLastError();
+    }
+    HeadArgs hh = h;
+    TailArgs tt = t;
+    unsigned *ticket = s.ticket;
+    int n_slots = p.n_slots, hid_bytes = p.hid_bytes, one = 1;
+    void *args[] = {&hh, &tt, &P, &ticket, &n_slots, &hid_bytes, &one};
+    e = launch_dependent((const void *)head_stream_kernel<RT, VR>, dim3((unsigned)grid), dim3(kThreads), p.smem, stream, args);
+    if (e != cudaSuccess) return e;
+    return launch_head_finalize(P, grid, h.R, h.n_rows_dev, t, s.ticket, sm_count, stream);
 }
 
 template <int RT>
 cudaError_t launch_rt(const HeadArgs &h, const TailArgs &t, const Scratch &s, const Plan &p, int grid,
-                      cudaStream_t stream)
+                      cudaStream_t stream, bool split_tail, int sm_count)
 {
     switch (p.VR) {
-        case 8:  return launch_inst<RT, 8>(h, t, s, p, grid, stream);
-        case 4:  return launch_inst<RT, 4>(h, t, s, p, grid, stream);
-        case 2:  return launch_inst<RT, 2>(h, t, s, p, grid, stream);
-        default: return launch_inst<RT, 1>(h, t, s, p, grid, stream);
+        case 8:  return launch_inst<RT, 8>(h, t, s, p, grid, stream, split_tail, sm_count);
+        case 4:  return launch_inst<RT, 4>(h, t, s, p, grid, stream, split_tail, sm_count);
+        case 2:  return launch_inst<RT, 2>(h, t, s, p, grid, stream, split_tail, sm_count);
+        default: return launch_inst<RT, 1>(h, t, s, p, grid, stream, split_tail, sm_count);
     }
 }
 
 }  // namespace
 
 cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch &s, int sm_count,
-                             cudaStream_t stream, int *launched)
+                             cudaStream_t stream, int *launched, bool split_tail)
 {
-    if (launched) *launched = 1;
+    if (launched) *launched = split_tail ? 2 : 1;
     Plan p = make_plan(h.R, h.d);
     if (p.n_slots < 1) return cudaErrorInvalidValue;
     int grid = sm_count;
@@ -292,9 +310,9 @@ cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch
     if (grid > kMaxSlices) grid = kMaxSlices;
     if (grid < 1) grid = 1;
     switch (p.RT) {
-        case 1:  return launch_rt<1>(h, t, s, p, grid, stream);
-        case 2:  return launch_rt<2>(h, t, s, p, grid, stream);
-        default: return launch_rt<4>(h, t, s, p, grid, stream);
+        case 1:  return launch_rt<1>(h, t, s, p, grid, stream, split_tail, sm_count);
+        case 2:  return launch_rt<2>(h, t, s, p, grid, stream, split_tail, sm_count);
+        default: return launch_rt<4>(h, t, s, p, grid, stream, split_tail, sm_count);
     }
 }
 

@@ -34,8 +34,9 @@ __host__ inline Scratch scratch_carve(void *ws)
 
 // CUDA-core streaming kernel: split-V GEMV for a handful of rows.
 // *launched (optional for the streaming kernel) receives the number of kernels enqueued.
+// split_tail: the kernel stops at the per-slice statistics and head_finalize_kernel is launched behind it.
 cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch &s, int sm_count,
-                             cudaStream_t stream, int *launched = nullptr);
+                             cudaStream_t stream, int *launched = nullptr, bool split_tail = false);
 
 // Tensor-core kernel (tcgen05 + tensor memory): any row count; the choice between the two is the
 // caller's.  gather_buf (umma_gather_bytes(R, d) bytes, 256-byte aligned) is used only with row_idx.
@@ -43,6 +44,13 @@ bool        umma_shape_ok(int R, int d, int V);
 size_t      umma_gather_bytes(int R, int d);
 cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
                              int sm_count, cudaStream_t stream, int *launched, bool use_pair);
+
+// The cross-block merge and the routing tail as a launch of its own, behind a head kernel that was
+// launched without its fused tail (rstitch_finalize.cu).  Both launches carry the programmatic stream
+// serialisation attribute; launch_dependent is the launch helper for such kernels.
+cudaError_t launch_dependent(const void *func, dim3 grid, dim3 block, size_t smem, cudaStream_t stream, void **args);
+cudaError_t launch_head_finalize(const Partials &P, int n_slices, int R, const int32_t *n_rows_dev,
+                                 const TailArgs &t, unsigned *ticket, int sm_count, cudaStream_t stream);
 
 // Merge of the gathered vocabulary shards ([n_shards][R][5] words, shard-major) and the routing tail.
 cudaError_t launch_shard_merge(const float *gathered, int n_shards, const int32_t *n_rows_dev, const TailArgs &t,

@@ -82,6 +82,22 @@ __device__ __forceinline__ void fence_proxy_async_all()
     asm volatile("fence.proxy.async;" ::: "memory");
 }
 
+// ---- programmatic dependent launch ------------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may begin while the kernel
+// before it in the stream is still running, once every block of that kernel has executed
+// launch_dependents (or exited).  What the earlier kernel wrote is visible only after wait, which
+// returns when that kernel has completed and flushed its memory; without a pending dependency both
+// instructions do nothing.
+__device__ __forceinline__ void grid_dep_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+__device__ __forceinline__ void grid_dep_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- bulk copies ------------------------------------------------------------------------
 // Untiled copy global -> shared; both addresses 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)

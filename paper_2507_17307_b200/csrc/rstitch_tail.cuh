@@ -143,57 +143,61 @@ __device__ inline void tail_finalize_rows(const Partials &P, int n_slices, const
     }
 }
 
-// Finalisation for a handful of rows and at most 256 slices: one warp per row pulls every partial of
-// the row into registers with all loads in flight at once (a single round trip to L2), then merges
-// without a dependent chain: the row maximum M and the greedy token first, then one exponential per
-// partial for the sums.
+// One row's n_slices <= 256 partials merged by one warp: every partial of the row is pulled into
+// registers with all loads in flight at once (a single round trip to L2), then merged without a
+// dependent chain: the row maximum M and the greedy token first, then one exponential per partial for
+// the sums.  Every lane returns the merged statistics.
+__device__ __forceinline__ Stats tail_row_direct(const Partials &P, size_t base, int n_slices, int lane)
+{
+    float m[8], s[8], u[8], bv[8];
+    int bi[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int c = lane + 32 * k;
+        const bool in = c < n_slices;
+        const size_t at = base + (in ? c : 0);
+        m[k]  = in ? __ldcg(P.m + at)  : -CUDART_INF_F;
+        s[k]  = in ? __ldcg(P.s + at)  : 0.f;
+        u[k]  = in ? __ldcg(P.u + at)  : 0.f;
+        bv[k] = in ? __ldcg(P.bv + at) : -CUDART_INF_F;
+        bi[k] = in ? __ldcg(P.bi + at) : INT_MAX;
+    }
+    float M = -CUDART_INF_F, best = -CUDART_INF_F;
+    int besti = INT_MAX;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { M = fmaxf(M, m[k]); argmax_take(best, besti, bv[k], bi[k]); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        float obv = __shfl_xor_sync(0xffffffffu, best, o);
+        int obi = __shfl_xor_sync(0xffffffffu, besti, o);
+        argmax_take(best, besti, obv, obi);
+    }
+    float ss = 0.f, uu = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+        if (m[k] != -CUDART_INF_F) {
+            const float dm = m[k] - M, e = __expf(dm);
+            ss = fmaf(e, s[k], ss);
+            uu = fmaf(e, fmaf(dm, s[k], u[k]), uu);
+        }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        uu += __shfl_xor_sync(0xffffffffu, uu, o);
+    }
+    Stats t;
+    t.m = M; t.s = ss; t.u = uu; t.bv = best; t.bi = besti;
+    return t;
+}
+
+// Finalisation for a handful of rows and at most 256 slices: one warp per row.
 __device__ inline void tail_finalize_rows_direct(const Partials &P, int n_slices, const TailArgs &a)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     for (int r = warp; r < a.R; r += nwarps) {
-        float m[8], s[8], u[8], bv[8];
-        int bi[8];
-        const size_t base = (size_t)r * n_slices;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int c = lane + 32 * k;
-            const bool in = c < n_slices;
-            const size_t at = base + (in ? c : 0);
-            m[k]  = in ? __ldcg(P.m + at)  : -CUDART_INF_F;
-            s[k]  = in ? __ldcg(P.s + at)  : 0.f;
-            u[k]  = in ? __ldcg(P.u + at)  : 0.f;
-            bv[k] = in ? __ldcg(P.bv + at) : -CUDART_INF_F;
-            bi[k] = in ? __ldcg(P.bi + at) : INT_MAX;
-        }
-        float M = -CUDART_INF_F, best = -CUDART_INF_F;
-        int besti = INT_MAX;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { M = fmaxf(M, m[k]); argmax_take(best, besti, bv[k], bi[k]); }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-            float obv = __shfl_xor_sync(0xffffffffu, best, o);
-            int obi = __shfl_xor_sync(0xffffffffu, besti, o);
-            argmax_take(best, besti, obv, obi);
-        }
-        float ss = 0.f, uu = 0.f;
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-            if (m[k] != -CUDART_INF_F) {
-                const float dm = m[k] - M, e = __expf(dm);
-                ss = fmaf(e, s[k], ss);
-                uu = fmaf(e, fmaf(dm, s[k], u[k]), uu);
-            }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            ss += __shfl_xor_sync(0xffffffffu, ss, o);
-            uu += __shfl_xor_sync(0xffffffffu, uu, o);
-        }
-        if (lane == 0) {
-            Stats t;
-            t.m = M; t.s = ss; t.u = uu; t.bv = best; t.bi = besti;
-            tail_emit_row(t, r, a);
-        }
+        const Stats t = tail_row_direct(P, (size_t)r * n_slices, n_slices, lane);
+        if (lane == 0) tail_emit_row(t, r, a);
     }
 }
 
