@@ -197,21 +197,27 @@ struct UmmaPlan {
 
 __global__ void __launch_bounds__(kThreads, 1)
 head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_constant__ WMaps tm_w,
-                 HeadArgs h, TailArgs t, Partials P, unsigned *ticket, UmmaPlan plan)
+                 HeadArgs h, TailArgs t, Partials P, UmmaPlan plan)
 {
+    // The kernels after this one in the stream (head_finalize_kernel, then the next call's head kernel) may be
+    // scheduled as soon as every block has got here; they wait for this kernel's completion themselves
+    // before they touch what it writes.
+    ptx::grid_dep_launch_dependents();
     extern __shared__ unsigned char dyn_smem_raw[];
     __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
     const int n_slices = plan.n_slices, n_stages = plan.n_stages;
-    __shared__ __align__(8) uint64_t s_acc_full[2], s_acc_empty[2], s_done, s_tailbar;
+    __shared__ __align__(8) uint64_t s_acc_full[2], s_acc_empty[2], s_done;
     __shared__ uint32_t s_tmem_base;
-    __shared__ int s_tail[66];
-    __shared__ int s_last, s_abort, s_zero;
+    __shared__ int s_abort, s_zero;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ring = (ptx::smem_u32(dyn_smem_raw) + 1023u) & ~1023u;
     const int nK = (h.d + kTileK - 1) / kTileK;
     int R_live = h.R;
-    if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
+    // A live row count on the device is the output of an earlier kernel: wait for it.  Without one the
+    // producer starts on W_head (a weight no earlier kernel writes) at once and waits only before its
+    // first copy of hidden rows.
+    if (h.n_rows_dev) { ptx::grid_dep_wait(); int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
 
     Schedule sch;
     sch.init(h.V, gridDim.x, blockIdx.x, plan.tiles_per_block);
@@ -228,7 +234,6 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
             ptx::mbar_init(ptx::smem_u32(&s_acc_empty[b]), kEpiWarps);   // one arrival per epilogue warp
         }
         ptx::mbar_init(ptx::smem_u32(&s_done), 1);
-        ptx::mbar_init(ptx::smem_u32(&s_tailbar), 1);
         ptx::mbar_fence_init();
         ptx::prefetch_tmap(&tm_hidden);
         ptx::prefetch_tmap(&tm_w.box[4]);
@@ -248,6 +253,19 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
         if (lane == 0) {
             int stage = 0, round = 0, issued = 0;
             bool live = true;
+            // The hidden rows may be the output of the kernel before this one, W_head is not.  Until the first
+            // pass over the ring is complete only the W parts of the stages are fetched, and the hidden
+            // tiles owed to those stages are remembered; then the producer waits for the earlier kernels,
+            // pays the debt and goes on with whole stages.  A ring of W_head is in flight meanwhile.
+            bool waited = (h.n_rows_dev != nullptr);
+            uint32_t owed_full[kMaxStages], owed_dst[kMaxStages];
+            int owed_x[kMaxStages], n_owed = 0;
+            auto settle = [&]() {
+                ptx::grid_dep_wait();
+                for (int q = 0; q < n_owed; ++q) ptx::tma_g2s_2d(owed_dst[q], &tm_hidden, owed_x[q], 0, owed_full[q]);
+                n_owed = 0;
+                waited = true;
+            };
             for (int j = 0; live && j < sch.n_items; ++j) {
                 const Item it = sch.item(j);
                 const uint32_t bytes = (uint32_t)((plan.a_rows + it.N) * kTileK * 2);
@@ -257,6 +275,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                 for (int ks = 0; live && ks < nK; ks += kIssueGroup) {
                     int ng = nK - ks < kIssueGroup ? nK - ks : kIssueGroup;
                     if (ng > n_stages) ng = n_stages;
+                    if (!waited && issued + ng > n_stages) settle();     // the ring has been round once
                     uint32_t full[kIssueGroup], a_dst[kIssueGroup];
                     for (int g = 0; g < ng; ++g) {
                         int sg = stage + g, rd = round;
@@ -273,8 +292,14 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                     }
                     // only the first a_rows rows of the hidden tile are fetched; the MMA reads all 128,
                     // and what the stale rows produce lands in accumulator rows nobody looks at
-                    for (int g = 0; g < ng; ++g)
-                        ptx::tma_g2s_2d(a_dst[g], &tm_hidden, (ks + g) * kTileK, 0, full[g]);
+                    for (int g = 0; g < ng; ++g) {
+                        if (waited) {
+                            ptx::tma_g2s_2d(a_dst[g], &tm_hidden, (ks + g) * kTileK, 0, full[g]);
+                        } else {
+                            owed_full[n_owed] = full[g]; owed_dst[n_owed] = a_dst[g]; owed_x[n_owed] = (ks + g) * kTileK;
+                            ++n_owed;
+                        }
+                    }
                     int r = 0;
 #pragma unroll
                     for (int b = 4; b >= 0; --b) {
@@ -292,6 +317,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                     if (ng < kIssueGroup && ks + ng < nK) ks += ng - kIssueGroup;   // fewer stages than a group
                 }
             }
+            if (!waited) settle();                   // fewer k-steps than stages: every armed stage gets its hidden tile
             if (s_abort && pid == 0) {
                 // no copy may still be landing in this block's shared memory when it exits
                 int first = issued > n_stages ? issued - n_stages : 0;
@@ -390,6 +416,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
             xch[slot + 4] = __int_as_float(st.bi);
         }
         asm volatile("bar.sync 1, %0;" :: "n"(kEpiWarps * 32) : "memory");
+        ptx::grid_dep_wait();                        // the scratch may still be read by the call before this one
         if (half == 0 && lane_has_row) {
             Stats o;
             o.m = xch[slot]; o.s = xch[slot + 1]; o.u = xch[slot + 2]; o.bv = xch[slot + 3];
@@ -400,35 +427,12 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     }
 
     ptx::tc_fence_before_sync();
-    __threadfence();
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
-    // the last block done merges all slices and runs the routing tail
-    if (threadIdx.x == 0) {
-        unsigned k = atomicAdd(ticket, 1u);
-        s_last = (k == (unsigned)(gridDim.x - 1));
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    TailArgs ta = t;
-    ta.R = R_live;
-    if (h.n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
-    // the ring is idle now: stage the partials through it (fast path), or read them from L2
-    if (ta.R > 8) {
-        unsigned char *stage = dyn_smem_raw + (ring - ptx::smem_u32(dyn_smem_raw));
-        if (!tail_finalize_rows_staged(P, n_slices, ta, stage, (uint32_t)kRingBytes, &s_tailbar, 0u, &s_abort) &&
-            threadIdx.x == 0)
-            raise_abort(&s_abort, t.stat, 0x205u);
-    } else {
-        tail_finalize_rows(P, n_slices, ta);
-    }
-    __syncthreads();
-    tail_route(ta, s_tail);
-    if (threadIdx.x == 0) *ticket = 0u;
+    // head_finalize_kernel, launched behind this kernel, merges the blocks' partials and decides
 }
 
 // ---- several M tiles, two per W tile ------------------------------------------------------------
@@ -532,6 +536,8 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ring = (ptx::smem_u32(dyn_smem_raw) + 1023u) & ~1023u;
     const int nK = (h.d + kTileK - 1) / kTileK;
+    ptx::grid_dep_launch_dependents();
+    ptx::grid_dep_wait();          // hidden rows, the live count and the scratch may come from the kernels before
     int R_live = h.R;
     if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
     const Sched2 sch = sched2_make(nM, h.V, (int)gridDim.x, (int)blockIdx.x, R_live > 0);
@@ -731,6 +737,8 @@ head_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __gri
     const uint32_t rank = ptx::cluster_ctarank();            // 0 = leader
     const uint32_t ring = (ptx::smem_u32(dyn_smem_raw) + 1023u) & ~1023u;
     const int nK = (h.d + kTileK - 1) / kTileK;
+    ptx::grid_dep_launch_dependents();
+    ptx::grid_dep_wait();          // hidden rows, the live count and the scratch may come from the kernels before
     int R_live = h.R;
     if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
     const int nG = (nM + 3) / 4;                             // groups of four M tiles
@@ -915,38 +923,6 @@ head_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __gri
     }
 }
 
-// Several M tiles: one warp per row merges that row's per-tile partials; the last block done
-// applies the rule and compacts.
-__global__ void __launch_bounds__(256)
-head_finalize_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_slices)
-{
-    __shared__ int s_tail[66];
-    __shared__ int s_last;
-    int R_live = h.R;
-    if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
-    const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (r < R_live) {
-        Stats st = tail_merge_strided(P, (size_t)r * n_slices, n_slices, lane, 32);
-        stats_warp_allmerge(st);
-        if (lane == 0) tail_emit_row(st, r, t);
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned k = atomicAdd(ticket, 1u);
-        s_last = (k == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    TailArgs ta = t;
-    ta.R = R_live;
-    if (h.n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
-    tail_route(ta, s_tail);
-    if (threadIdx.x == 0) *ticket = 0u;
-}
-
 // hidden[row_idx[r]] -> packed[r] (zero for rows past the live count or with a bad index).
 __global__ void __launch_bounds__(128)
 gather_rows_kernel(HeadArgs h, uint4 *packed, int rows_padded, DevStat *stat)
@@ -1081,9 +1057,12 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
     if (!make_map(&tm_h, hid_base, hid_rows, h.d, plan.a_rows)) return cudaErrorInvalidValue;
     for (int b = 0; b < 5; ++b)
         if (!make_map(&tm_w.box[b], h.W, h.V, h.d, 16 << b)) return cudaErrorInvalidValue;
+    Partials Pk = P;
+    HeadArgs hk2 = hk;
+    TailArgs tk = t;
     if (plan.nM == 1) {
-        head_umma_kernel<<<grid, kThreads, kDynSmem, stream>>>(tm_h, tm_w, hk, t, P, s.ticket, plan);
-        e = cudaGetLastError();
+        void *args[] = {&tm_h, &tm_w, &hk2, &tk, &Pk, &plan};
+        e = launch_dependent((const void *)head_umma_kernel, dim3((unsigned)grid), dim3(kThreads), kDynSmem, stream, args);
     } else if (use_pair && grid >= 2) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(grid & ~1));
@@ -1097,15 +1076,12 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
         cfg.numAttrs = 1;
         e = cudaLaunchKernelEx(&cfg, head_umma_pair_kernel, tm_h, tm_w, hk, t, P, plan.nM, plan.n_slices);
     } else {
-        head_umma2_kernel<<<grid, kThreads2, kDynSmem2, stream>>>(tm_h, tm_w, hk, t, P, plan.nM, plan.n_slices);
-        e = cudaGetLastError();
+        void *args[] = {&tm_h, &tm_w, &hk2, &tk, &Pk, &plan.nM, &plan.n_slices};
+        e = launch_dependent((const void *)head_umma2_kernel, dim3((unsigned)grid), dim3(kThreads2), kDynSmem2, stream, args);
     }
     if (e != cudaSuccess) return e;
     ++*launched;
-    if (plan.nM == 1) return e;
-    const int fin_grid = (h.R + 7) / 8;
-    head_finalize_kernel<<<fin_grid, 256, 0, stream>>>(hk, t, P, s.ticket, plan.n_slices);
-    e = cudaGetLastError();
+    e = launch_head_finalize(P, plan.n_slices, h.R, hk.n_rows_dev, t, s.ticket, sm_count, stream);
     if (e == cudaSuccess) ++*launched;
     return e;
 }
