@@ -115,7 +115,7 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a, ValidateMode mo
         if (a->n_src < 0) return RSTITCH_ERR_INVALID_ARG;
         if ((a->flags & RSTITCH_PATH_GEMV) && (a->flags & RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
         if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA |
-                         RSTITCH_PATH_PAIR | RSTITCH_PATH_FUSED_TAIL))
+                         RSTITCH_PATH_PAIR))
             return RSTITCH_ERR_INVALID_ARG;
         if ((a->flags & RSTITCH_SAMPLE) && !(std::isfinite(a->temperature) && a->temperature > 0.f))
             return RSTITCH_ERR_INVALID_ARG;
@@ -135,7 +135,7 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a, ValidateMode mo
         if (a->R > kMaxRows) return RSTITCH_ERR_UNSUPPORTED_SHAPE;
         if (!std::isfinite(a->tau)) return RSTITCH_ERR_INVALID_ARG;
         if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA |
-                         RSTITCH_PATH_PAIR | RSTITCH_PATH_FUSED_TAIL))
+                         RSTITCH_PATH_PAIR))
             return RSTITCH_ERR_INVALID_ARG;
         if (!a->llm_count) return RSTITCH_ERR_INVALID_ARG;
         if (a->row_seq == nullptr && a->B != a->R) return RSTITCH_ERR_INVALID_ARG;
@@ -157,7 +157,7 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a, ValidateMode mo
     if (!std::isfinite(a->tau)) return RSTITCH_ERR_INVALID_ARG;
     if ((a->flags & RSTITCH_PATH_GEMV) && (a->flags & RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
     if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA |
-                     RSTITCH_PATH_PAIR | RSTITCH_PATH_FUSED_TAIL))
+                     RSTITCH_PATH_PAIR))
         return RSTITCH_ERR_INVALID_ARG;
     if ((a->flags & RSTITCH_SAMPLE) && !(std::isfinite(a->temperature) && a->temperature > 0.f))
         return RSTITCH_ERR_INVALID_ARG;
@@ -285,7 +285,7 @@ int enqueue_head(rstitch_handle_s *h, const rstitch_args_t *a, cudaStream_t stre
         e = launch_head_umma(ha, ta, sc, (char *)ws + kWsHeader + part, h->sm_count, stream, &launched,
                              (a->flags & RSTITCH_PATH_PAIR) != 0);
     } else {
-        e = launch_head_gemv(ha, ta, sc, h->sm_count, stream, &launched, !(a->flags & RSTITCH_PATH_FUSED_TAIL));
+        e = launch_head_gemv(ha, ta, sc, h->sm_count, stream, &launched);
     }
     h->launch_count += (unsigned)launched;
     if (e != cudaSuccess) { cudaGetLastError(); return RSTITCH_ERR_CUDA; }

@@ -17,12 +17,18 @@ namespace {
 
 constexpr int kFinThreads = 128;
 constexpr int kFinRows    = kFinThreads / 32;        // one warp per row
+constexpr int kFinStageSeqs = 128;                   // mask bytes the deciding block keeps in shared memory
 
 __global__ void __launch_bounds__(kFinThreads)
 head_finalize_kernel(Partials P, int n_slices, int R, const int32_t *n_rows_dev, TailArgs t, unsigned *ticket)
 {
     __shared__ int s_tail[66];
     __shared__ int s_last;
+    // Shared memory is kept to a few hundred bytes on purpose: a block of this kernel has to fit on an SM
+    // beside a block of a head kernel, which leaves about 1.5 KB; if it does not, it takes the SM of the
+    // first head block to finish and keeps the next call's block off that SM until the whole merge is done.
+    __shared__ float s_ent[kFinRows];                // one block only: its rows' entropies stay on the SM
+    __shared__ uint8_t s_mask[kFinStageSeqs];        // the mask, for the compaction
     ptx::grid_dep_launch_dependents();
     ptx::grid_dep_wait();                            // the head kernel has completed: its partials are visible
     int R_live = R;
@@ -36,7 +42,10 @@ head_finalize_kernel(Partials P, int n_slices, int R, const int32_t *n_rows_dev,
             st = tail_merge_strided(P, (size_t)r * n_slices, n_slices, lane, 32);
             stats_warp_allmerge(st);
         }
-        if (lane == 0) tail_emit_row(st, r, t);
+        if (lane == 0) {
+            const float H = tail_emit_row(st, r, t);
+            if (r < kFinRows) s_ent[r] = H;
+        }
     }
     if (gridDim.x > 1) {
         __threadfence();
@@ -54,7 +63,10 @@ head_finalize_kernel(Partials P, int n_slices, int R, const int32_t *n_rows_dev,
     TailArgs ta = t;
     ta.R = R_live;
     if (n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
-    tail_route(ta, s_tail);
+    // what this block can keep on the SM it does not read back from global memory: the entropies when
+    // it merged every row itself, the mask whenever it fits
+    tail_route(ta, s_tail, (gridDim.x == 1 && ta.R <= kFinRows) ? s_ent : nullptr,
+               ta.B <= kFinStageSeqs ? s_mask : nullptr);
     if (gridDim.x > 1 && threadIdx.x == 0) *ticket = 0u;
 }
 

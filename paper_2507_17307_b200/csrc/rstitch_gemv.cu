@@ -44,17 +44,15 @@ __device__ __forceinline__ void raise_abort(volatile int *flag, DevStat *stat, u
 // RT hidden rows per pass, VR vocabulary rows per ring slot.
 template <int RT, int VR>
 __global__ void __launch_bounds__(kThreads, 1)
-head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_slots, int hid_bytes, int split_tail)
+head_stream_kernel(HeadArgs h, TailArgs t, Partials P, int n_slots, int hid_bytes)
 {
-    // split_tail: the merge of the slices and the routing tail run in head_finalize_kernel, launched
-    // behind this kernel; the next call's kernel may start as soon as this one's blocks leave their SMs.
-    if (split_tail) ptx::grid_dep_launch_dependents();
+    // The merge of the slices and the routing tail run in head_finalize_kernel, launched behind this
+    // kernel; it and the next call's head kernel may be scheduled as soon as every block has got here.
+    ptx::grid_dep_launch_dependents();
     extern __shared__ __align__(128) unsigned char dyn_smem[];   // [hidden RT x d][ring]
     __shared__ __align__(8) uint64_t s_full[kMaxSlots];
     __shared__ __align__(8) uint64_t s_empty[kMaxSlots];
     __shared__ Stats s_warp[kConsumerWarps][RT];
-    __shared__ int   s_tail[66];
-    __shared__ int   s_last;
     __shared__ int   s_abort;
     __shared__ int   s_zero;
 
@@ -212,25 +210,6 @@ head_stream_kernel(HeadArgs h, TailArgs t, Partials P, unsigned *ticket, int n_s
             ptx::mbar_wait(ptx::smem_u32(&s_full[j % n_slots]), (uint32_t)((j / n_slots) & 1), &s_zero);
     }
 
-    if (split_tail) return;                    // head_finalize_kernel merges the slices and decides
-    // last block done: merge all slices and run the routing tail
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned k = atomicAdd(ticket, 1u);
-        s_last = (k == (unsigned)(n_slices - 1));
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    TailArgs ta = t;
-    ta.R = R_live;
-    if (h.n_rows_dev) ta.B = R_live < t.B ? R_live : t.B;
-    if (n_slices <= 256 && ta.R <= 2 * (kThreads / 32)) tail_finalize_rows_direct(P, n_slices, ta);
-    else                                                tail_finalize_rows(P, n_slices, ta);
-    __syncthreads();
-    tail_route(ta, s_tail);
-    if (threadIdx.x == 0) *ticket = 0u;
 }
 
 struct Plan { int RT, VR, n_slots, hid_bytes; size_t smem; };
@@ -257,7 +236,7 @@ Plan make_plan(int R, int d)
 
 template <int RT, int VR>
 cudaError_t launch_inst(const HeadArgs &h, const TailArgs &t, const Scratch &s, const Plan &p, int grid,
-                        cudaStream_t stream, bool split_tail, int sm_count)
+                        cudaStream_t stream, int sm_count)
 {
     static bool configured[64] = {};
     int dev = 0;
@@ -270,15 +249,10 @@ cudaError_t launch_inst(const HeadArgs &h, const TailArgs &t, const Scratch &s, 
         configured[dev] = true;
     }
     Partials P = partials_carve(s.partials, (size_t)h.R, (size_t)grid);
-    if (!split_tail) {
-        head_stream_kernel<RT, VR><<<grid, kThreads, p.smem, stream>>>(h, t, P, s.ticket, p.n_slots, p.hid_bytes, 0);
-        return cudaGetLastError();
-    }
     HeadArgs hh = h;
     TailArgs tt = t;
-    unsigned *ticket = s.ticket;
-    int n_slots = p.n_slots, hid_bytes = p.hid_bytes, one = 1;
-    void *args[] = {&hh, &tt, &P, &ticket, &n_slots, &hid_bytes, &one};
+    int n_slots = p.n_slots, hid_bytes = p.hid_bytes;
+    void *args[] = {&hh, &tt, &P, &n_slots, &hid_bytes};
     e = launch_dependent((const void *)head_stream_kernel<RT, VR>, dim3((unsigned)grid), dim3(kThreads), p.smem, stream, args);
     if (e != cudaSuccess) return e;
     return launch_head_finalize(P, grid, h.R, h.n_rows_dev, t, s.ticket, sm_count, stream);
@@ -286,22 +260,22 @@ cudaError_t launch_inst(const HeadArgs &h, const TailArgs &t, const Scratch &s, 
 
 template <int RT>
 cudaError_t launch_rt(const HeadArgs &h, const TailArgs &t, const Scratch &s, const Plan &p, int grid,
-                      cudaStream_t stream, bool split_tail, int sm_count)
+                      cudaStream_t stream, int sm_count)
 {
     switch (p.VR) {
-        case 8:  return launch_inst<RT, 8>(h, t, s, p, grid, stream, split_tail, sm_count);
-        case 4:  return launch_inst<RT, 4>(h, t, s, p, grid, stream, split_tail, sm_count);
-        case 2:  return launch_inst<RT, 2>(h, t, s, p, grid, stream, split_tail, sm_count);
-        default: return launch_inst<RT, 1>(h, t, s, p, grid, stream, split_tail, sm_count);
+        case 8:  return launch_inst<RT, 8>(h, t, s, p, grid, stream, sm_count);
+        case 4:  return launch_inst<RT, 4>(h, t, s, p, grid, stream, sm_count);
+        case 2:  return launch_inst<RT, 2>(h, t, s, p, grid, stream, sm_count);
+        default: return launch_inst<RT, 1>(h, t, s, p, grid, stream, sm_count);
     }
 }
 
 }  // namespace
 
 cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch &s, int sm_count,
-                             cudaStream_t stream, int *launched, bool split_tail)
+                             cudaStream_t stream, int *launched)
 {
-    if (launched) *launched = split_tail ? 2 : 1;
+    if (launched) *launched = 2;
     Plan p = make_plan(h.R, h.d);
     if (p.n_slots < 1) return cudaErrorInvalidValue;
     int grid = sm_count;
@@ -310,9 +284,9 @@ cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch
     if (grid > kMaxSlices) grid = kMaxSlices;
     if (grid < 1) grid = 1;
     switch (p.RT) {
-        case 1:  return launch_rt<1>(h, t, s, p, grid, stream, split_tail, sm_count);
-        case 2:  return launch_rt<2>(h, t, s, p, grid, stream, split_tail, sm_count);
-        default: return launch_rt<4>(h, t, s, p, grid, stream, split_tail, sm_count);
+        case 1:  return launch_rt<1>(h, t, s, p, grid, stream, sm_count);
+        case 2:  return launch_rt<2>(h, t, s, p, grid, stream, sm_count);
+        default: return launch_rt<4>(h, t, s, p, grid, stream, sm_count);
     }
 }
 

@@ -34,9 +34,10 @@ __host__ inline Scratch scratch_carve(void *ws)
 
 // CUDA-core streaming kernel: split-V GEMV for a handful of rows.
 // *launched (optional for the streaming kernel) receives the number of kernels enqueued.
-// split_tail: the kernel stops at the per-slice statistics and head_finalize_kernel is launched behind it.
+// Both head launchers enqueue the head kernel, which stops at the per-slice statistics, and
+// head_finalize_kernel behind it.
 cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch &s, int sm_count,
-                             cudaStream_t stream, int *launched = nullptr, bool split_tail = false);
+                             cudaStream_t stream, int *launched = nullptr);
 
 // Tensor-core kernel (tcgen05 + tensor memory): any row count; the choice between the two is the
 // caller's.  gather_buf (umma_gather_bytes(R, d) bytes, 256-byte aligned) is used only with row_idx.

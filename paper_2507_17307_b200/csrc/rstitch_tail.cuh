@@ -1,6 +1,7 @@
-// Cross-CTA finalisation of the head kernels and the routing tail (S2-S6), run by ONE thread
-// block: the block that drew the last ticket of a head kernel, or the single block of the
-// stand-alone compaction kernel.  No block ever waits on another, so nothing here can hang.
+// Cross-block merge of the head kernels' partial statistics and the routing tail (S2-S6).  The merge is
+// one warp per row (head_finalize_kernel); the tail is run by ONE thread block: the block of that kernel
+// (or of the shard-merge kernel) that drew the last ticket, or the single block of the stand-alone
+// compaction kernel.  No block ever waits on another, so nothing here can hang.
 #pragma once
 #include "rstitch_stats.cuh"
 #include "rstitch_ptx.cuh"
@@ -80,21 +81,22 @@ struct TailArgs {
 
 constexpr int kShardWords = 5;
 
-// Writes ent_out / tok_out of one row from its merged statistics.
-__device__ __forceinline__ void tail_emit_row(const Stats &t, int r, const TailArgs &a)
+// Writes ent_out / tok_out of one row from its merged statistics; returns the entropy.
+__device__ __forceinline__ float tail_emit_row(const Stats &t, int r, const TailArgs &a)
 {
     if (a.shard_stats) {
         float *o = a.shard_stats + (size_t)r * kShardWords;
         const bool found = !(t.bi == INT_MAX || t.bi < 0 || t.bi >= a.V);
         o[0] = t.m; o[1] = t.s; o[2] = t.u; o[3] = t.bv;
         o[4] = __int_as_float(found ? t.bi + a.v_base : INT_MAX);
-        return;
+        return 0.f;
     }
     float H = logf(t.s) - t.u / t.s;
     if (H < 0.f) H = 0.f;                      // rounding below zero; NaN stays NaN
     a.ent_out[r] = H;
     a.tok_out[r] = (t.bi == INT_MAX || t.bi < 0 || t.bi >= a.V) ? 0 : t.bi;
     if (H != H) atomicAdd(&a.stat->nan_rows, 1u);
+    return H;
 }
 
 // Merge of slices part, part + parts, ... of one row by one thread, loads issued four at a time.
@@ -118,29 +120,6 @@ __device__ __forceinline__ Stats tail_merge_strided(const Partials &P, size_t ro
         stats_merge(t, p);
     }
     return t;
-}
-
-// Merge the n_slices partials of every row in a fixed order and write ent_out / tok_out.  A row is
-// shared by `parts` adjacent lanes (a power of two, as many as the block can spare for the row
-// count), each taking a strided subset of the slices; a butterfly over the group finishes the row.
-__device__ inline void tail_finalize_rows(const Partials &P, int n_slices, const TailArgs &a)
-{
-    int parts = 32;
-    while (parts > 1 && a.R * parts > (int)blockDim.x) parts >>= 1;
-    const int rows_per_pass = (int)blockDim.x / parts;
-    const int part = threadIdx.x & (parts - 1);
-    const int sub = threadIdx.x / parts;
-    const bool in_pass = sub < rows_per_pass;          // blockDim.x need not be a multiple of parts
-    for (int r0 = 0; r0 < a.R; r0 += rows_per_pass) {
-        const int r = r0 + sub;
-        const bool act = in_pass && r < a.R;
-        Stats t = act ? tail_merge_strided(P, (size_t)r * n_slices, n_slices, part, parts) : stats_empty();
-        for (int o = parts >> 1; o > 0; o >>= 1) {     // whole warp takes part: same trip count everywhere
-            Stats p = stats_shfl_xor(t, o);
-            stats_merge(t, p);
-        }
-        if (act && part == 0) tail_emit_row(t, r, a);
-    }
 }
 
 // One row's n_slices <= 256 partials merged by one warp: every partial of the row is pulled into
@@ -191,121 +170,35 @@ __device__ __forceinline__ Stats tail_row_direct(const Partials &P, size_t base,
     return t;
 }
 
-// Finalisation for a handful of rows and at most 256 slices: one warp per row.
-__device__ inline void tail_finalize_rows_direct(const Partials &P, int n_slices, const TailArgs &a)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    for (int r = warp; r < a.R; r += nwarps) {
-        const Stats t = tail_row_direct(P, (size_t)r * n_slices, n_slices, lane);
-        if (lane == 0) tail_emit_row(t, r, a);
-    }
-}
-
-// The same finalisation for many rows (tensor-core kernel, up to 128 rows x ~150 slices), where
-// fetching the partials straight from L2 is a chain of dependent round trips.  The partials of a
-// group of rows are first brought into shared memory with five bulk copies (one per statistics
-// array; the rows of a group are contiguous in each), then merged from there without a dependent
-// chain: pass 1 takes the row maximum M and the greedy token, pass 2 sums e^{m_i - M} s_i and
-// e^{m_i - M} (u_i + (m_i - M) s_i), one exponential per partial.
-//   stage / stage_bytes: free shared memory (16-byte aligned); bar: an initialised mbarrier
-//   (count 1) whose completed phases so far number bar_phase.
-// Returns false if a bounded wait ran out (the caller records it).
-__device__ inline bool tail_finalize_rows_staged(const Partials &P, int n_slices, const TailArgs &a,
-                                                 unsigned char *stage, uint32_t stage_bytes, uint64_t *bar,
-                                                 uint32_t bar_phase, volatile int *abort_flag)
-{
-    int parts = 32;
-    while (parts > 1 && a.R * parts > (int)blockDim.x) parts >>= 1;
-    const int part = threadIdx.x & (parts - 1);
-    const int sub = threadIdx.x / parts;
-    const uint32_t row_bytes = (uint32_t)n_slices * 4u;
-    int group = stage_bytes > 80u ? (int)((stage_bytes - 80u) / 5u / row_bytes) & ~3 : 0;   // rows per group
-    if (group > (int)blockDim.x / parts) group = ((int)blockDim.x / parts) & ~3;
-    if (group < 4) {                                                     // no room to stage: read from L2
-        tail_finalize_rows(P, n_slices, a);
-        return true;
-    }
-    const uint32_t region = (((uint32_t)group * row_bytes + 15u) & ~15u);
-    const float *sm_m = (const float *)(stage);
-    const float *sm_s = (const float *)(stage + region);
-    const float *sm_u = (const float *)(stage + 2 * region);
-    const float *sm_bv = (const float *)(stage + 3 * region);
-    const int   *sm_bi = (const int *)(stage + 4 * region);
-    const uint32_t bar_u32 = ptx::smem_u32(bar);
-    bool ok = true;
-    for (int g0 = 0; g0 < a.R; g0 += group, ++bar_phase) {
-        const int rows = (a.R - g0) < group ? (a.R - g0) : group;
-        if (threadIdx.x == 0) {
-            const uint32_t bytes = (((uint32_t)rows * row_bytes + 15u) & ~15u);
-            const size_t off = (size_t)g0 * n_slices;
-            ptx::fence_proxy_async_all();       // the partials were written with ordinary stores
-            ptx::mbar_arrive_expect_tx(bar_u32, 5u * bytes);
-            ptx::bulk_g2s(ptx::smem_u32(sm_m), P.m + off, bytes, bar_u32);
-            ptx::bulk_g2s(ptx::smem_u32(sm_s), P.s + off, bytes, bar_u32);
-            ptx::bulk_g2s(ptx::smem_u32(sm_u), P.u + off, bytes, bar_u32);
-            ptx::bulk_g2s(ptx::smem_u32(sm_bv), P.bv + off, bytes, bar_u32);
-            ptx::bulk_g2s(ptx::smem_u32(sm_bi), P.bi + off, bytes, bar_u32);
-        }
-        if (!ptx::mbar_wait(bar_u32, bar_phase & 1u, abort_flag)) ok = false;
-        const int r = g0 + sub;
-        const bool act = ok && sub < rows;
-        const int base = sub * n_slices;
-        float M = -CUDART_INF_F, bv = -CUDART_INF_F;
-        int bi = INT_MAX;
-        if (act)
-            for (int c = part; c < n_slices; c += parts) {
-                M = fmaxf(M, sm_m[base + c]);
-                argmax_take(bv, bi, sm_bv[base + c], sm_bi[base + c]);
-            }
-        for (int o = parts >> 1; o > 0; o >>= 1) {
-            M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-            float obv = __shfl_xor_sync(0xffffffffu, bv, o);
-            int obi = __shfl_xor_sync(0xffffffffu, bi, o);
-            argmax_take(bv, bi, obv, obi);
-        }
-        float ss = 0.f, uu = 0.f;
-        if (act)
-            for (int c = part; c < n_slices; c += parts) {
-                const float mi = sm_m[base + c];
-                if (mi != -CUDART_INF_F) {
-                    const float dm = mi - M, e = __expf(dm), si = sm_s[base + c];
-                    ss = fmaf(e, si, ss);
-                    uu = fmaf(e, fmaf(dm, si, sm_u[base + c]), uu);
-                }
-            }
-        for (int o = parts >> 1; o > 0; o >>= 1) {
-            ss += __shfl_xor_sync(0xffffffffu, ss, o);
-            uu += __shfl_xor_sync(0xffffffffu, uu, o);
-        }
-        if (act && part == 0) {
-            Stats t;
-            t.m = M; t.s = ss; t.u = uu; t.bv = bv; t.bi = bi;
-            tail_emit_row(t, r, a);
-        }
-        __syncthreads();                        // the stage is reused by the next group
-    }
-    return ok;
-}
-
 // Eq. 2 / Algorithm 1: mask = H > tau (strict); a NaN entropy routes to the LLM.
 __device__ __forceinline__ uint8_t rule(float H, float tau)
 {
     return (H != H || H > tau) ? 1 : 0;
 }
 
-// S4: per-sequence mask from per-row entropies already in global memory (written by this block).
-__device__ inline void tail_mask(const TailArgs &a)
+// S4: per-sequence mask from the per-row entropies: ent is a.ent_out (global memory, written before the
+// block's last barrier) or the block's own copy of it in shared memory.  With mask_stage (shared memory,
+// a.B bytes) the mask is also kept there for the compaction, which then reads nothing back from global.
+__device__ inline void tail_mask(const TailArgs &a, const float *ent, uint8_t *mask_stage)
 {
     if (a.row_seq == nullptr) {
-        for (int b = threadIdx.x; b < a.B; b += blockDim.x)
-            a.route_mask[b] = (b < a.R) ? rule(a.ent_out[b], a.tau) : 0;
+        for (int b = threadIdx.x; b < a.B; b += blockDim.x) {
+            const uint8_t m = (b < a.R) ? rule(ent[b], a.tau) : 0;
+            a.route_mask[b] = m;
+            if (mask_stage) mask_stage[b] = m;
+        }
     } else {
-        for (int b = threadIdx.x; b < a.B; b += blockDim.x) a.route_mask[b] = 0;
+        uint8_t *mk = mask_stage ? mask_stage : a.route_mask;
+        for (int b = threadIdx.x; b < a.B; b += blockDim.x) mk[b] = 0;
         __syncthreads();
         for (int r = threadIdx.x; r < a.R; r += blockDim.x) {
             int sq = a.row_seq[r];
             bool last = (r == a.R - 1) || (a.row_seq[r + 1] != sq);
-            if (last && sq >= 0 && sq < a.B) a.route_mask[sq] = rule(a.ent_out[r], a.tau);
+            if (last && sq >= 0 && sq < a.B) mk[sq] = rule(ent[r], a.tau);
+        }
+        if (mask_stage) {
+            __syncthreads();
+            for (int b = threadIdx.x; b < a.B; b += blockDim.x) a.route_mask[b] = mask_stage[b];
         }
     }
     __syncthreads();
@@ -368,12 +261,12 @@ __device__ inline void tail_compact(const uint8_t *mask, int B, const int32_t *s
 
 // S4-S6 for at most 32 sequences decided row by row: one warp, ballots and shuffles, no block barrier.
 // The entropies were written by this block before its last barrier.
-__device__ inline void tail_route_warp(const TailArgs &a)
+__device__ inline void tail_route_warp(const TailArgs &a, const float *ent)
 {
     if (threadIdx.x >= 32) return;
     const int b = threadIdx.x;
     const bool in = b < a.B;
-    const bool routed = in && b < a.R && rule(a.ent_out[b], a.tau) != 0;
+    const bool routed = in && b < a.R && rule(ent[b], a.tau) != 0;
     if (in) a.route_mask[b] = routed ? 1 : 0;
     const unsigned ball = __ballot_sync(0xffffffffu, routed);
     const int rank = __popc(ball & ((1u << b) - 1u));
@@ -402,15 +295,19 @@ __device__ inline void tail_route_warp(const TailArgs &a)
     }
 }
 
-__device__ inline void tail_route(const TailArgs &a, int *smem)
+// ent_stage / mask_stage (optional, shared memory): the block's own copy of the a.R entropies it has just
+// written, and room for a.B mask bytes; without them both are read back from global memory.
+__device__ inline void tail_route(const TailArgs &a, int *smem, const float *ent_stage = nullptr,
+                                  uint8_t *mask_stage = nullptr)
 {
     if (a.shard_stats) return;                       // a vocabulary shard decides nothing
+    const float *ent = ent_stage ? ent_stage : a.ent_out;
     if (a.B <= 32 && a.row_seq == nullptr) {
-        tail_route_warp(a);
+        tail_route_warp(a, ent);
     } else {
-        tail_mask(a);
-        tail_compact(a.route_mask, a.B, a.seq_len, a.kv_len, a.llm_idx, a.llm_count, a.llm_span,
-                     a.llm_row_off, a.stat, smem);
+        tail_mask(a, ent, mask_stage);
+        tail_compact(mask_stage ? mask_stage : a.route_mask, a.B, a.seq_len, a.kv_len, a.llm_idx, a.llm_count,
+                     a.llm_span, a.llm_row_off, a.stat, smem);
     }
     if (a.alg1.on) alg1_tail_block(a.alg1, a.tok_out, a.route_mask, smem);
     if (a.mirror_dst) {
