@@ -162,12 +162,18 @@ def recorded_traffic(workload: str):
 # ------------------------------------------------------------------------------------------
 # workload state
 # ------------------------------------------------------------------------------------------
+_W_CACHE = {}
+
+
 def build_batches(names, n_rot: int, rank: int):
     """Host-side synthetic inputs: per head its W bits and n_rot rotating hidden batches."""
     heads = []
     for name in names:
         w = gen.WORKLOADS[name]
-        w_bits = gen.make_w_head(w)
+        key = (w.seed, w.d, w.V, w.sigma_w)
+        if key not in _W_CACHE:                 # workloads that share a head draw it once
+            _W_CACHE[key] = gen.make_w_head(w)
+        w_bits = _W_CACHE[key]
         batches = []
         for i in range(n_rot):
             step = rank * 100003 + i
@@ -350,58 +356,59 @@ def run_vocab_parallel(args, names, rank, local_rank, world) -> int:
     return 0
 
 
-def main() -> int:
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None)
-    ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="c2_slm_b1", choices=sorted(BENCH_WORKLOADS))
-    ap.add_argument("--impl", default="native", choices=["native", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="rstitch_args_t.flags (testing)")
-    ap.add_argument("--graph", action="store_true",
-                    help="capture one rotation of steps into a CUDA graph and time its replays")
-    ap.add_argument("--vocab-parallel", action="store_true",
-                    help="shard W_head by vocabulary rows over the ranks instead of the batch by rows")
-    args = ap.parse_args()
+def free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+        sk.bind(("127.0.0.1", 0))
+        return int(sk.getsockname()[1])
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    names = BENCH_WORKLOADS[args.workload]
 
-    if args.impl == "reference":
-        if rank != 0:
-            return 0
-        args.steps = 8 if args.steps is None else args.steps
-        args.warmup = 1 if args.warmup is None else args.warmup
-        print(json.dumps(run_reference(args, names)), flush=True)
-        return 0
+def needs_spawn(gpus: int, env) -> bool:
+    """--gpus N > 1 without a launcher's environment: this process starts the N ranks itself."""
+    return gpus > 1 and "WORLD_SIZE" not in env and "RANK" not in env
 
-    if args.vocab_parallel:
-        return run_vocab_parallel(args, names, rank, local_rank, world)
 
-    import torch
-    import paper_2507_17307_b200 as rs
-    from paper_2507_17307_b200 import build as rs_build
-    if rank == 0:
-        rs_build.build_library()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-        dist.barrier()
-    rs.lib()
+def default_steps(workload: str):
+    """(steps, warm-up, rotating buffers) when the command line leaves them open."""
+    if workload == "c5_catchup":
+        return 64, 3, 2
+    if workload in ("c4_batched", "alg1_b64"):
+        return 2048, 64, 8
+    return 8192, 64, 8
 
-    heavy = args.workload in ("c5_catchup",)
-    K = args.steps if args.steps is not None else (64 if heavy else (2048 if args.workload in ("c4_batched", "alg1_b64") else 8192))
-    Wm = args.warmup if args.warmup is not None else (3 if heavy else 64)
-    Wm = max(Wm, 3)
-    n_rot = 2 if heavy else 8
 
+def read_stream_ceiling(rs, torch, dev, stream) -> dict:
+    """Bandwidth of a read-only pass over 2 GiB with the streaming head kernel's own copy pipeline."""
+    n = 2 << 30
+    buf = torch.empty(n, dtype=torch.uint8, device=dev)
+    buf.zero_()
+    gave_up = torch.zeros(1, dtype=torch.int32, device=dev)
+    for _ in range(3):
+        rs.probe_read_stream(buf, gave_up, stream=stream)
+    torch.cuda.synchronize()
+    best, times = None, []
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        rs.probe_read_stream(buf, gave_up, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    if int(gave_up.item()) != 0:
+        return {"gbs": None, "note": "a bounded wait ran out: no figure"}
+    del buf
+    torch.cuda.empty_cache()
+    ms = float(np.median(times))
+    return {"gbs": n / (ms / 1e3) / 1e9, "gbs_best": n / (min(times) / 1e3) / 1e9, "bytes": n,
+            "how": "rstitch_probe_read_stream: 148 blocks, bulk copies into a shared-memory ring, nothing written; "
+                   "median of 10 passes, CUDA events"}
+
+
+def measure(rs, torch, dist, rank, local_rank, world, args, workload: str, K: int, Wm: int, n_rot: int,
+            with_e2e: bool, min_region_s: float = 0.2) -> dict:
+    """Build one workload on this rank's GPU, time `repeats` regions of exactly K steps each with CUDA
+    events on the launching stream, and (with_e2e) the same steps through the host-buffer entry point."""
+    names = BENCH_WORKLOADS[workload]
     heads = build_batches(names, n_rot, rank)
     dev = torch.device("cuda", local_rank)
 
@@ -412,7 +419,7 @@ def main() -> int:
         return None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
 
     stream = torch.cuda.current_stream()
-    alg1 = args.workload == "alg1_b64"
+    alg1 = workload == "alg1_b64"
     state = None
     if alg1:
         B0 = gen.WORKLOADS[names[0]].B
@@ -421,7 +428,7 @@ def main() -> int:
         # fitted coefficients printed in the paper's latency-regression appendix (SLM-1.5B, LLM-7B), ms
         lat_models = [rs.LatencyModel(0.000021, 0.000231, -0.121046, 27.090929),
                       rs.LatencyModel(0.000027, 0.000031, -0.045256, 27.040801)]
-    with_router = args.workload == "c4_router"
+    with_router = workload == "c4_router"
     router = None
     if with_router:
         d0 = gen.WORKLOADS[names[0]].d
@@ -466,7 +473,6 @@ def main() -> int:
         flops += 2.0 * np.mean([b["R"] for b in h["batches"]]) * w.d * w.V
     w0 = heads[0]["w"]
     rows_per_step = float(np.mean([b["R"] for b in heads[0]["batches"]]))
-    decisions_per_step = rows_per_step            # rows decided by the first head of the step
 
     if alg1:
         # the first round's plans; every later round is planned by the LLM call of the round before
@@ -490,10 +496,6 @@ def main() -> int:
     warm_launches = sum(rs.last_status(hd)["launches"] for hd in handles)     # also clears the counters
     launches_per_step = warm_launches / float(Wm) + (1 if with_router else 0)
 
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
     graph = None
     if args.graph:
         # the step loop has no host synchronisation, so a whole rotation of steps records into one graph
@@ -502,11 +504,11 @@ def main() -> int:
         cap_stream.wait_stream(stream)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.stream(cap_stream):
-            saved = stream
-            stream = cap_stream
             for calls in prepared:
                 for c in calls:
                     c._stream = int(cap_stream.cuda_stream)
+            saved = stream
+            stream = cap_stream
             with torch.cuda.graph(graph, stream=cap_stream):
                 for i in range(n_rot):
                     step(i)
@@ -520,7 +522,9 @@ def main() -> int:
         torch.cuda.synchronize()
         for hd in handles:
             rs.last_status(hd)
-    with ClockSampler(visible_gpu_index(local_rank)) as clocks:
+
+    def region():
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record(torch.cuda.current_stream())
         if graph is not None:
             for _ in range(K // n_rot):
@@ -530,15 +534,43 @@ def main() -> int:
                 step(i)
         ev1.record(torch.cuda.current_stream())
         torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1)
+
+    # every region times exactly K steps; regions are repeated until they add up to min_region_s
+    # (at least three), the step time reported is the median region's
     if dist is not None:
         dist.barrier()
-    ms = ev0.elapsed_time(ev1)
+    torch.cuda.synchronize()
+    times = []
+    with ClockSampler(visible_gpu_index(local_rank)) as clocks:
+        total = 0.0
+        while len(times) < 3 or (total < min_region_s * 1e3 and len(times) < 400):
+            ms_r = region()
+            times.append(ms_r)
+            total += ms_r
+    if dist is not None:
+        dist.barrier()
+    repeats = n_run = len(times)
+    if dist is not None and world > 1:
+        # every rank runs the same number of regions: the fewest any rank chose
+        t = torch.tensor([repeats], dtype=torch.int64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MIN)
+        repeats = int(t.item())
+        times = times[:repeats]
+    ms = float(np.median(times))
     stats = [rs.last_status(hd) for hd in handles]
-    launches = sum(st["launches"] for st in stats) + (1 * K if with_router else 0)
-    if graph is not None:
-        launches = int(round(K * launches_per_step))      # replayed kernels are not counted by the handles
+    launches_all = sum(st["launches"] for st in stats) + (n_run * K if with_router else 0)
+    launches = int(round(launches_all / float(n_run))) if graph is None else int(round(K * launches_per_step))
     if any(st["timeouts"] or st["nan_rows"] for st in stats):
         raise SystemExit("device status after the timed region: %s" % stats)
+
+    res = {"workload": workload, "names": names, "heads": heads, "K": K, "Wm": Wm, "n_rot": n_rot, "ms": ms,
+           "ms_min": float(min(times)), "ms_max": float(max(times)), "repeats": repeats, "launches": launches,
+           "clocks": clocks.summary(), "algo_bytes": algo_bytes, "flops": flops, "rows_per_step": rows_per_step,
+           "w0": w0, "handles": handles, "dev": dev,
+           "path": [rs.path_name(int(rows_per_step), h["w"].d, h["w"].V, args.flags) for h in heads]}
+    if not with_e2e:
+        return res
 
     # end to end: the same step through rstitch_route_ex_host -- every per-step input starts in pinned
     # host memory, every output lands in host memory, copies and the stream synchronisation are inside
@@ -606,88 +638,204 @@ def main() -> int:
                 if st != 0:
                     raise rs.RstitchError(st, "rstitch_route_ex_host")
 
-    Ke = max(1, min(K, 2048 if not heavy else 32))
+    Ke = max(1, min(K, 2048 if workload != "c5_catchup" else 32))
     for i in range(3):
         host_step(i)
     torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    t0 = time.perf_counter()
-    for i in range(Ke):
-        host_step(i)
-    torch.cuda.synchronize()
-    e2e = {"seconds": time.perf_counter() - t0, "steps": Ke, "h2d": h2d, "d2h": d2h}
+    e2e_times = []
+    reps_e = 3 if Ke >= 256 else max(3, min(50, int(0.1 / max(1e-6, Ke * ms / K / 1e3))))
+    for _ in range(reps_e):
+        if dist is not None:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for i in range(Ke):
+            host_step(i)
+        torch.cuda.synchronize()
+        e2e_times.append(time.perf_counter() - t0)
+    res["e2e"] = {"seconds": float(np.median(e2e_times)), "steps": Ke, "h2d": h2d, "d2h": d2h, "repeats": reps_e}
     for hd in handles:
         rs.last_status(hd)
+    return res
+
+
+def roofline_of(res: dict, peaks: dict, read_gbs) -> dict:
+    per_step_s = res["ms"] / 1e3 / res["K"]
+    if res["rows_per_step"] >= 256:
+        achieved = res["flops"] / per_step_s / 1e12
+        long_run = res["ms"] > 1000.0
+        peak = peaks["bf16_tflops_sustained"] if long_run else peaks["bf16_tflops"]
+        return {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "traffic": recorded_traffic(res["workload"]), "peak_source": "of " + peaks["source"] +
+                (" (sustained figure: the timed region exceeds 1 s)" if long_run else " (burst figure)"),
+                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                "hbm_gbs": res["algo_bytes"] / per_step_s / 1e9}
+    achieved = res["algo_bytes"] / per_step_s / 1e9
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved / peaks["hbm_gbs"], "traffic": recorded_traffic(res["workload"]),
+            "peak_source": "of " + peaks["source"] + " (copy: reads + writes)",
+            "frac_of_8tbs_nominal": achieved / 8000.0, "tflops": res["flops"] / per_step_s / 1e12}
+    if read_gbs:
+        roof["read_stream_gbs"] = read_gbs
+        roof["frac_of_read_stream"] = achieved / read_gbs
+    return roof
+
+
+def release(res: dict, torch):
+    for hd in res["handles"]:
+        hd.destroy()
+    for h in res["heads"]:
+        h.pop("w_dev", None)
+    res["heads"] = None
+    torch.cuda.empty_cache()
+
+
+EXTRA_WORKLOADS = ("c3_llm_b1", "c3_llm_b4", "c3_llm_b16", "c4_slm_b64", "c4_batched", "c5_catchup")
+
+
+def main() -> int:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default=None, choices=sorted(BENCH_WORKLOADS),
+                    help="default: c2_slm_b1 as the headline, the other configurations beside it under 'workloads'")
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="only the headline workload")
+    ap.add_argument("--flags", type=lambda s: int(s, 0), default=0, help="rstitch_args_t.flags (testing)")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture one rotation of steps into a CUDA graph and time its replays")
+    ap.add_argument("--vocab-parallel", action="store_true",
+                    help="shard W_head by vocabulary rows over the ranks instead of the batch by rows")
+    args = ap.parse_args()
+
+    if args.impl != "reference" and needs_spawn(args.gpus, os.environ):
+        # no launcher around this process: start one rank per GPU here, same command line
+        from paper_2507_17307_b200 import sharding
+        return sharding.spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:])
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    extras = args.workload is None and not args.no_extras and world == 1 and not args.graph and args.flags == 0
+    if args.workload is None:
+        args.workload = "c2_slm_b1"
+    names = BENCH_WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        args.steps = 8 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        print(json.dumps(run_reference(args, names)), flush=True)
+        return 0
+
+    if args.vocab_parallel:
+        return run_vocab_parallel(args, names, rank, local_rank, world)
+
+    import torch
+    import paper_2507_17307_b200 as rs
+    from paper_2507_17307_b200 import build as rs_build, sharding
+    if rank == 0:
+        rs_build.build_library()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    rs.lib()
+    dev = torch.device("cuda", local_rank)
+
+    dK, dW, n_rot = default_steps(args.workload)
+    K = args.steps if args.steps is not None else dK
+    Wm = max(args.warmup if args.warmup is not None else dW, 3)
+    res = measure(rs, torch, dist, rank, local_rank, world, args, args.workload, K, Wm, n_rot, with_e2e=True)
+    K = res["K"]
 
     # max over ranks of the times, sums of the rest
-    from paper_2507_17307_b200 import sharding
-    ms, _, launches = sharding.reduce_step_stats(ms, decisions_per_step, launches, dist, dev)
+    ms, _, launches = sharding.reduce_step_stats(res["ms"], res["rows_per_step"], res["launches"], dist, dev)
+    ms_min, _, _ = sharding.reduce_step_stats(res["ms_min"], 0.0, 0, dist, dev)
+    ms_max, _, _ = sharding.reduce_step_stats(res["ms_max"], 0.0, 0, dist, dev)
+    e2e = res["e2e"]
     e2e["seconds"], _, _ = sharding.reduce_step_stats(e2e["seconds"], 0.0, 0, dist, dev)
+    res["ms"] = ms
 
     if rank == 0:
         peaks = measured_peaks()
+        read = read_stream_ceiling(rs, torch, dev, torch.cuda.current_stream()) if world == 1 else {"gbs": None}
         sec = ms / 1e3
-        value = world * decisions_per_step * K / sec
-        per_launch_s = sec / K
-        tensor_bound = rows_per_step >= 256
-        if tensor_bound:
-            achieved = flops / per_launch_s / 1e12
-            peak = peaks["bf16_tflops_sustained"] if sec > 1.0 else peaks["bf16_tflops"]
-            roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                    "frac": achieved / peak, "traffic": recorded_traffic(args.workload),
-                    "peak_source": "of " + peaks["source"],
-                    "hbm_gbs": algo_bytes / per_launch_s / 1e9}
-        else:
-            achieved = algo_bytes / per_launch_s / 1e9
-            roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": recorded_traffic(args.workload),
-                    "peak_source": "of " + peaks["source"], "frac_of_8tbs_nominal": achieved / 8000.0,
-                    "tflops": flops / per_launch_s / 1e12}
+        w0, alg1 = res["w0"], args.workload == "alg1_b64"
+        value = world * res["rows_per_step"] * K / sec
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "B": w0.B, "rows_per_step": rows_per_step, "d": w0.d,
-                       "V": w0.V, "tau_nats": w0.tau_nats, "heads": list(names),
-                       "path": [rs.path_name(int(rows_per_step), h["w"].d, h["w"].V, args.flags) for h in heads],
+            "config": {"workload": args.workload, "B": w0.B, "rows_per_step": res["rows_per_step"], "d": w0.d,
+                       "V": w0.V, "tau_nats": w0.tau_nats, "heads": list(names), "path": res["path"],
                        "l2": "inputs larger than L2: each step streams the whole W_head (%.0f MB); "
-                             "hidden rotates over %d buffers" % (algo_bytes / 1e6, n_rot),
+                             "hidden rotates over %d buffers" % (res["algo_bytes"] / 1e6, n_rot),
                        "parallelism": "dp%d (rows sharded, head replicated, no collective)" % world,
                        "cuda_graph": bool(args.graph)},
-            "roofline": roof, "clocks": clocks.summary(), "gpu_launches": launches,
-            "algorithmic_bytes_per_step": algo_bytes, "flops_per_step": flops,
+            "timing": {"regions": res["repeats"], "steps_per_region": K, "statistic": "median region",
+                       "ms_per_step_min": ms_min / K, "ms_per_step_max": ms_max / K,
+                       "note": "every region times exactly `steps` steps between two CUDA events on the launching "
+                               "stream; regions repeat until they add up to 0.2 s (at least three)"},
+            "roofline": roofline_of(res, peaks, read.get("gbs")), "clocks": res["clocks"], "gpu_launches": launches,
+            "algorithmic_bytes_per_step": res["algo_bytes"], "flops_per_step": res["flops"],
             # `value` counts rows (every row gets a token and an entropy); with multi-row spans a sequence
             # is decided by its last row, so the sequences decided per second are fewer
             "rows_per_s": value, "sequences_per_s": world * w0.B * K / sec,
         }
-        line["e2e"] = {"value": world * decisions_per_step * e2e["steps"] / e2e["seconds"], "unit": UNIT,
+        if read.get("gbs"):
+            line["read_stream"] = read
+        line["e2e"] = {"value": world * res["rows_per_step"] * e2e["steps"] / e2e["seconds"], "unit": UNIT,
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                       "steps": e2e["steps"],
+                       "steps": e2e["steps"], "regions": e2e["repeats"],
                        "note": ("the round's hidden pools copied from pinned host memory, per-sequence token counts "
                                 "copied back, stream synchronised every round; W_head resident") if alg1 else
                                ("rstitch_route_ex_host: pinned hidden and index arrays in, tok/ent/mask/llm_idx/"
                                 "llm_count/spans out, stream synchronised every step; W_head resident")}
+        heads_for_cpu = res["heads"]
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
             budget, t0, rows, n = 12.0, time.perf_counter(), 0, 0
-            sample_rows = 8 if rows_per_step > 16 else None
+            sample_rows = 8 if res["rows_per_step"] > 16 else None
             while time.perf_counter() - t0 < budget and n < 4096:
-                for h in heads:
+                for h in heads_for_cpu:
                     b = h["batches"][n % n_rot]
                     hid = b["hid"] if sample_rows is None else b["hid"][:sample_rows]
                     oracle.route(hid, h["w_bits"], h["w"].tau_nats)
-                rows += (heads[0]["batches"][n % n_rot]["hid"].shape[0] if sample_rows is None else sample_rows)
+                rows += (heads_for_cpu[0]["batches"][n % n_rot]["hid"].shape[0] if sample_rows is None else sample_rows)
                 n += 1
             dt = time.perf_counter() - t0
             line["cpu_baseline"] = {"value": rows / dt, "unit": UNIT, "cores": oracle.num_threads(),
                                     "kind": "oracle",
                                     "sample": "%d steps%s of the same batches, %.1f s" % (
                                         n, "" if sample_rows is None else " (first %d rows each)" % sample_rows, dt)}
+        release(res, torch)
+        if extras:
+            # the other configurations, each in a short timed region of its own with its own clock record
+            line["workloads"] = {}
+            for wl in EXTRA_WORKLOADS:
+                eK, eW, e_rot = default_steps(wl)
+                eK = args.steps if args.steps is not None else min(eK, 512)
+                r = measure(rs, torch, None, 0, local_rank, 1, args, wl, eK, max(3, min(Wm, 8)), e_rot, with_e2e=False)
+                per_step_s = r["ms"] / 1e3 / r["K"]
+                line["workloads"][wl] = {
+                    "ms_per_step": r["ms"] / r["K"], "ms_per_step_min": r["ms_min"] / r["K"],
+                    "ms_per_step_max": r["ms_max"] / r["K"], "regions": r["repeats"], "steps_per_region": r["K"],
+                    "rows_per_step": r["rows_per_step"], "rows_per_s": r["rows_per_step"] / per_step_s,
+                    "d": r["w0"].d, "V": r["w0"].V, "heads": list(r["names"]), "path": r["path"],
+                    "gpu_launches": r["launches"], "roofline": roofline_of(r, peaks, read.get("gbs")),
+                    "clocks": r["clocks"]}
+                release(r, torch)
         print(json.dumps(line), flush=True)
-    for hd in handles:
-        hd.destroy()
+    else:
+        release(res, torch)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()

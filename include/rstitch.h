@@ -394,6 +394,17 @@ int rstitch_last_status(rstitch_handle_t h, rstitch_devstat_t *out);
 #define RSTITCH_SELFTEST_SITE 0x7e57u
 int rstitch_selftest_wait(rstitch_handle_t h, void *cuda_stream);
 
+/*
+ * Measurement aid (not part of the routing path): one pass over buf [bytes] (device, 16-byte aligned) that
+ * only reads it, through the pipeline of the streaming head kernel (one block per SM, bulk copies of a
+ * contiguous slice into a shared-memory ring) with nothing done to the bytes.  Timed by the caller with
+ * CUDA events it gives the bandwidth ceiling of a read-only stream on this GPU, the regime of the head
+ * kernels at small batch (Section 3.1's last linear map read once per step), beside the usual copy
+ * figure.  Whole 16 KiB chunks are read; a remainder is skipped.  *gave_up (device, zeroed by the
+ * caller) counts bounded waits that ran out, which voids the measurement.
+ */
+int rstitch_probe_read_stream(const void *buf, size_t bytes, uint32_t *gave_up, void *cuda_stream);
+
 /* Static, never NULL. */
 const char *rstitch_status_string(int status);
 

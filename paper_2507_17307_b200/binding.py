@@ -125,6 +125,8 @@ def lib():
         L.rstitch_path_name.restype = C.c_char_p
         L.rstitch_route_static.argtypes = [vp, vp, i, i, i, f, vp, vp, vp, vp, vp, vp]
         L.rstitch_route_static.restype = i
+        L.rstitch_probe_read_stream.argtypes = [vp, C.c_size_t, vp, vp]
+        L.rstitch_probe_read_stream.restype = i
         L.rstitch_selftest_wait.argtypes = [vp, vp]
         L.rstitch_selftest_wait.restype = i
         L.rstitch_shard_stats.argtypes = [vp, C.POINTER(_Args), C.c_int32, vp, vp]
@@ -462,6 +464,15 @@ def compact(mask, idx=None, count=None, stream=None):
 
 
 SELFTEST_SITE = 0x7E57
+
+
+def probe_read_stream(buf, gave_up, stream=None) -> int:
+    """One read-only pass over a device buffer (measurement aid); gave_up: zeroed uint32/int32 tensor [1]."""
+    st = lib().rstitch_probe_read_stream(_ptr(buf), buf.numel() * buf.element_size(), _ptr(gave_up),
+                                         _stream_ptr(stream))
+    if st != 0:
+        raise RstitchError(st, "rstitch_probe_read_stream")
+    return st
 
 
 def selftest_wait(handle: Handle, stream=None) -> int:

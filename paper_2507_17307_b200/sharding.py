@@ -14,7 +14,10 @@ CUDA tensors with NCCL.
 """
 from __future__ import annotations
 
-from typing import Tuple
+import os
+import socket
+import subprocess
+from typing import List, Optional, Tuple
 
 
 def rank_rows(n_rows: int, rank: int, world: int) -> Tuple[int, int]:
@@ -94,3 +97,50 @@ def gather_shard_stats(stats, dist=None, out=None):
     # the ranks' blocks concatenated along the first axis: the form every backend accepts
     dist.all_gather_into_tensor(out.view((world * stats.shape[0],) + tuple(stats.shape[1:])), stats.contiguous())
     return out
+
+
+def spawn_ranks(n_ranks: int, argv: List[str], port: Optional[int] = None, extra_env: Optional[dict] = None,
+                timeout: Optional[float] = None) -> int:
+    """Run the command line `argv` as n_ranks processes of one node, one per GPU, with the environment
+    torch.distributed reads (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR = 127.0.0.1, MASTER_PORT): what a
+    launcher would do, for callers that were started without one.  The ranks inherit stdout and stderr.
+    Returns 0 if every rank exited 0, else the first non-zero exit code; once a rank has failed the others
+    are terminated (by process id) instead of being left waiting at a rendezvous."""
+    if n_ranks < 1:
+        raise ValueError("n_ranks must be at least 1")
+    if port is None:
+        with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = int(sk.getsockname()[1])
+    procs = []
+    for r in range(n_ranks):
+        env = dict(os.environ)
+        env.update({"RANK": str(r), "LOCAL_RANK": str(r), "WORLD_SIZE": str(n_ranks), "LOCAL_WORLD_SIZE": str(n_ranks),
+                    "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+        if extra_env:
+            env.update(extra_env)
+        procs.append(subprocess.Popen(list(argv), env=env))
+    import time
+    deadline = None if timeout is None else time.monotonic() + timeout
+    rc = 0
+    pending = list(procs)
+    while pending:
+        for p in list(pending):
+            code = p.poll()
+            if code is not None:
+                pending.remove(p)
+                if code != 0 and rc == 0:
+                    rc = code
+        if rc != 0 or (deadline is not None and time.monotonic() > deadline):
+            for p in pending:
+                p.terminate()
+            for p in pending:
+                try:
+                    p.wait(timeout=10)
+                except subprocess.TimeoutExpired:
+                    p.kill()
+            if rc == 0:
+                rc = 124
+            break
+        time.sleep(0.05)
+    return rc
