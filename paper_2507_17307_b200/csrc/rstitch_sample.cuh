@@ -55,9 +55,9 @@ __device__ __forceinline__ float gumbel_from_bits(uint32_t x)
         p = fmaf(p, y2, 1.0f);
         t = 2.0f * y * p;
     } else {
-        t = -__logf(u);
+        t = -log_approx(u);
     }
-    return -__logf(t);
+    return -log_approx(t);
 }
 
 // Score of vocabulary entry v (any v): one generator call per entry.

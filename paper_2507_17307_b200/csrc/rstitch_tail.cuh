@@ -156,7 +156,7 @@ __device__ __forceinline__ Stats tail_row_direct(const Partials &P, size_t base,
 #pragma unroll
     for (int k = 0; k < 8; ++k)
         if (m[k] != -CUDART_INF_F) {
-            const float dm = m[k] - M, e = __expf(dm);
+            const float dm = m[k] - M, e = exp_approx(dm);
             ss = fmaf(e, s[k], ss);
             uu = fmaf(e, fmaf(dm, s[k], u[k]), uu);
         }

@@ -103,7 +103,7 @@ __device__ __forceinline__ void fold_chunk_full(Stats &st, const float (&z)[32],
     if (st.m == -CUDART_INF_F) { st.s = 0.f; st.u = 0.f; }
     else {
         float dm = st.m - m_new;
-        float a = __expf(dm);
+        float a = exp_approx(dm);
         st.u = a * (st.u + dm * st.s);
         st.s = a * st.s;
     }
@@ -112,7 +112,7 @@ __device__ __forceinline__ void fold_chunk_full(Stats &st, const float (&z)[32],
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
         float d0 = z[i] - m_new, d1 = z[i + 1] - m_new, d2 = z[i + 2] - m_new, d3 = z[i + 3] - m_new;
-        float e0 = __expf(d0), e1 = __expf(d1), e2 = __expf(d2), e3 = __expf(d3);   // NaN logit -> NaN sums
+        float e0 = exp_approx(d0), e1 = exp_approx(d1), e2 = exp_approx(d2), e3 = exp_approx(d3);   // NaN logit -> NaN sums
         s0 += e0; s1 += e1; s2 += e2; s3 += e3;
         u0 = fmaf(e0, d0, u0); u1 = fmaf(e1, d1, u1); u2 = fmaf(e2, d2, u2); u3 = fmaf(e3, d3, u3);
     }
@@ -153,7 +153,7 @@ __device__ __forceinline__ void fold_chunk_tail(Stats &st, const float (&z)[32],
     if (st.m == -CUDART_INF_F) { st.s = 0.f; st.u = 0.f; }
     else {
         float dm = st.m - m_new;
-        float a = __expf(dm);
+        float a = exp_approx(dm);
         st.u = a * (st.u + dm * st.s);
         st.s = a * st.s;
     }
@@ -163,7 +163,7 @@ __device__ __forceinline__ void fold_chunk_tail(Stats &st, const float (&z)[32],
     for (int i = 0; i < 32; ++i) {
         if (i < n_valid) {
             float dz = z[i] - m_new;
-            float e = __expf(dz);
+            float e = exp_approx(dz);
             s += e;
             u = fmaf(e, dz, u);
             const float sc = sa.on ? sample_score(sa, z[i], row, (uint32_t)(vbase + i)) : z[i];
