@@ -74,7 +74,8 @@ def _load():
         lib.oracle_latency_ms.argtypes = [f64p, c.c_int32, c.c_int32]
         lib.oracle_latency_ms.restype = c.c_double
         lib.oracle_alg1_sequence.argtypes = [c.c_int32, c.c_int32, c.c_double, c.c_int32, i32p, f64p, i32p, f64p,
-                                             f64p, f64p, i32p, i32p, i32p, i32p, i32p, f64p, i32p, i32p, i32p, i32p]
+                                             f64p, f64p, u8p, i32p, i32p, i32p, i32p, i32p, f64p, i32p, i32p, i32p,
+                                             i32p]
         lib.oracle_alg1_sequence.restype = None
         _lib = lib
     return _lib
@@ -211,8 +212,10 @@ def latency_ms(coef, n_inf: int, n_kv: int) -> float:
 
 
 def alg1_sequence(prompt_len: int, t_max: int, tau: float, eos_id: int, tok_slm, ent_slm, tok_llm, ent_llm,
-                  coef_slm, coef_llm) -> dict:
-    """Algorithm 1 for one sequence over recorded (token, entropy) streams of the two models."""
+                  coef_slm, coef_llm, switch_slm=None) -> dict:
+    """Algorithm 1 for one sequence over recorded (token, entropy) streams of the two models.
+    switch_slm (optional uint8 [t_max]): the router's decision per loop index (R-Stitch+), consulted
+    only when the SLM's entropy exceeds tau; None is R-Stitch (always switch)."""
     ts = np.ascontiguousarray(tok_slm, dtype=np.int32)
     tl = np.ascontiguousarray(tok_llm, dtype=np.int32)
     es = np.ascontiguousarray(ent_slm, dtype=np.float64)
@@ -220,6 +223,10 @@ def alg1_sequence(prompt_len: int, t_max: int, tau: float, eos_id: int, tok_slm,
     assert min(ts.size, tl.size, es.size, el.size) >= t_max
     cs = np.ascontiguousarray(coef_slm, dtype=np.float64)
     cl = np.ascontiguousarray(coef_llm, dtype=np.float64)
+    sw = None
+    if switch_slm is not None:
+        sw = np.ascontiguousarray(switch_slm, dtype=np.uint8)
+        assert sw.size >= t_max
     y = np.full(max(t_max, 1), -1, dtype=np.int32)
     i32 = lambda n=1: np.zeros(n, dtype=np.int32)
     n_out, active, L, ln, kept, steps, done, iters = i32(), i32(), i32(2), i32(), i32(2), i32(2), i32(), i32()
@@ -227,7 +234,7 @@ def alg1_sequence(prompt_len: int, t_max: int, tau: float, eos_id: int, tok_slm,
     P = lambda a: _p(a, ctypes.c_int32)
     D = lambda a: _p(a, ctypes.c_double)
     _load().oracle_alg1_sequence(int(prompt_len), int(t_max), float(tau), int(eos_id), P(ts), D(es), P(tl), D(el),
-                                 D(cs), D(cl), P(y), P(n_out), P(active), P(L), P(ln), D(lat), P(kept), P(steps),
+                                 D(cs), D(cl), _p(sw, ctypes.c_uint8), P(y), P(n_out), P(active), P(L), P(ln), D(lat), P(kept), P(steps),
                                  P(done), P(iters))
     n = int(n_out[0])
     return {"y": y[:n].copy(), "n_out": n, "active": int(active[0]), "L_slm": int(L[0]), "L_llm": int(L[1]),

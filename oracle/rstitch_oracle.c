@@ -231,11 +231,15 @@ double oracle_latency_ms(const double *coef, int32_t n_inf, int32_t n_kv)
  *     if L[active] < |x + y|:  prefill on (x + y)[L[active]:]  -> n_inf = |x + y| - L[active],
  *                              n_kv = L[active];  L[active] <- |x + y| + 1
  *     else:                    decode -> n_inf = 1, n_kv = L[active];  L[active] <- L[active] + 1
- *     H_t > tau:   (R-Stitch: switch = true)
- *        active == SLM: discard y_t, roll KV^SLM back by the one entry just added, active <- LLM, continue
- *        active == LLM: keep decoding on the LLM
+ *     H_t > tau:   switch = true (R-Stitch), or the router's decision for this step (R-Stitch+:
+ *                  switch = (argmax_a pi(a | s_t) == LLM), recorded in switch_slm[t]; NULL means R-Stitch)
+ *        active == SLM and switch: discard y_t, roll KV^SLM back by the one entry just added,
+ *                                  active <- LLM, continue
+ *        otherwise (SLM without switch, or LLM): the active model stays and y_t is kept
  *     else if active == LLM: active <- SLM
  *     append y_t;  stop after appending EOS
+ * The router is consulted only when H_t > tau and only changes what an SLM step does: low-entropy tokens
+ * always stay with the SLM, and on the LLM the rule is the entropy test alone.
  *
  * The latency estimate sums Eq. 5 over every model step taken, discarded ones included.
  *
@@ -246,7 +250,7 @@ double oracle_latency_ms(const double *coef, int32_t n_inf, int32_t n_kv)
 void oracle_alg1_sequence(int32_t prompt_len, int32_t t_max, double tau, int32_t eos_id,
                           const int32_t *tok_slm, const double *ent_slm,
                           const int32_t *tok_llm, const double *ent_llm,
-                          const double *coef_slm, const double *coef_llm,
+                          const double *coef_slm, const double *coef_llm, const uint8_t *switch_slm,
                           int32_t *y, int32_t *n_out, int32_t *active_out, int32_t *L_out,
                           int32_t *len_out, double *lat_ms, int32_t *kept, int32_t *steps,
                           int32_t *done, int32_t *iters)
@@ -277,11 +281,12 @@ void oracle_alg1_sequence(int32_t prompt_len, int32_t t_max, double tau, int32_t
         int32_t yt = active == 0 ? tok_slm[t] : tok_llm[t];
         const int gen = active;             /* the model that produced y_t */
         if (oracle_rule(H, tau)) {
-            if (active == 0) {              /* SLM -> LLM: token not kept */
+            const int sw = switch_slm ? (switch_slm[t] != 0) : 1;
+            if (active == 0 && sw) {        /* SLM -> LLM: token not kept */
                 L[0] -= 1;                  /* roll back the cache entry this step added */
                 active = 1;
                 continue;
-            }                               /* on the LLM: keep decoding with the LLM */
+            }                               /* the router kept the SLM, or the LLM keeps decoding */
         } else if (active == 1) {
             active = 0;                     /* LLM -> SLM */
         }

@@ -134,3 +134,59 @@ def test_alg1_against_second_simulation(oracle):
         assert r["kept_slm"] + r["kept_llm"] == r["n_out"] == r["len"] - P
         assert r["L_slm"] <= r["len"] and r["L_llm"] <= r["len"]
         assert r["steps_slm"] + r["steps_llm"] == r["iters"]
+
+
+# ---- Algorithm 1, the R-Stitch+ lines: switch <- (argmax_a pi(a | s_t) = LLM), consulted when H_t > tau ----
+
+def test_alg1_router_switch_worked_example(oracle):
+    # prompt of 4 tokens, tau = 0.5.  The SLM is unsure at loop indices 1, 2 and 4; the router keeps the
+    # SLM at 1, hands over at 2 (that token is discarded), the LLM stays unsure once and hands back at 4,
+    # where the SLM is unsure again and the router keeps it.
+    #   t      0     1     2       3          4       5
+    #   model  SLM   SLM   SLM->   LLM        LLM->   SLM
+    #   H      0.1   0.9   0.9     0.9        0.2     0.9
+    #   switch -     0     1       (ignored)  -       0
+    ts, es = [1, 2, 3, 4, 5, 6], [0.1, 0.9, 0.9, 0.0, 0.0, 0.9]
+    tl, el = [11, 12, 13, 14, 15, 16], [9.0, 9.0, 9.0, 0.9, 0.2, 9.0]
+    sw = [1, 0, 1, 0, 1, 0]          # entries at t = 0, 3, 4 must not matter
+    r = oracle.alg1_sequence(4, 6, 0.5, 99, ts, es, tl, el, (0, 0, 0, 1), (0, 0, 0, 10), switch_slm=sw)
+    assert r["y"].tolist() == [1, 2, 14, 15, 6]
+    assert (r["kept_slm"], r["kept_llm"], r["steps_slm"], r["steps_llm"]) == (3, 2, 4, 2)
+    # the LLM prefilled x + y = 4 + 2 tokens at t = 3, decoded at t = 4; the SLM prefilled its two missing
+    # tokens at t = 5
+    assert r["L_llm"] == 8 and r["L_slm"] == 9 and r["len"] == 9 and r["active"] == 0
+    assert r["lat_ms"] == 4 * 1.0 + 2 * 10.0
+    for flip in (0, 3, 4):           # the router is not consulted there
+        s2 = list(sw)
+        s2[flip] ^= 1
+        r2 = oracle.alg1_sequence(4, 6, 0.5, 99, ts, es, tl, el, (0, 0, 0, 1), (0, 0, 0, 10), switch_slm=s2)
+        assert r2["y"].tolist() == r["y"].tolist() and r2["lat_ms"] == r["lat_ms"]
+
+
+def test_alg1_router_switch_limits(oracle):
+    rng = random.Random(11)
+    c = coeffs()
+    for trial in range(100):
+        T, P = rng.randint(1, 50), rng.randint(1, 200)
+        tau = rng.choice([0.1, 0.3, 1.0])
+        ts = [rng.randint(0, 50) for _ in range(T)]
+        tl = [rng.randint(0, 50) for _ in range(T)]
+        es = [rng.choice([0.0, tau, tau + 1e-9, 2.0]) for _ in range(T)]
+        el = [rng.choice([0.0, tau, tau + 1e-9, 2.0]) for _ in range(T)]
+        args = (P, T, tau, -1, ts, es, tl, el, c["SLM-1.5B"], c["LLM-7B"])
+        # switch always true is R-Stitch
+        plain = oracle.alg1_sequence(*args)
+        always = oracle.alg1_sequence(*args, switch_slm=[1] * T)
+        assert always["y"].tolist() == plain["y"].tolist() and always["lat_ms"] == plain["lat_ms"]
+        assert (always["L_slm"], always["L_llm"], always["active"]) == (plain["L_slm"], plain["L_llm"], plain["active"])
+        # switch never true: the SLM decodes alone whatever its entropy (one prefill, then decodes)
+        never = oracle.alg1_sequence(*args, switch_slm=[0] * T)
+        assert never["y"].tolist() == ts and never["steps_llm"] == 0 and never["kept_llm"] == 0
+        assert never["active"] == 0 and never["L_llm"] == 0 and never["L_slm"] == P + T
+        # a random router never hands over more often than R-Stitch at the same threshold would let it:
+        # every LLM step follows an SLM step with H > tau and switch = 1
+        sw = [rng.randint(0, 1) for _ in range(T)]
+        mixed = oracle.alg1_sequence(*args, switch_slm=sw)
+        handoffs = mixed["steps_slm"] - mixed["kept_slm"]
+        assert handoffs <= sum(1 for t in range(T) if es[t] > tau and sw[t])
+        assert mixed["kept_slm"] + mixed["kept_llm"] == mixed["n_out"] and mixed["steps_slm"] + mixed["steps_llm"] == mixed["iters"]
