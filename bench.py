@@ -43,6 +43,10 @@ BENCH_WORKLOADS = {
     # launches: the SLM head on the sequences decoding on the SLM, the LLM head on the others, each applying
     # Algorithm 1's decision block in its own tail, the LLM's call also planning the next round
     "alg1_b64": ("c4_slm_b64", "c4_llm_b64"),
+    # the same round with Algorithm 1's R-Stitch+ lines, three launches: the SLM head (no decision block), the
+    # router on the rows above the threshold, whose last block refines the mask and runs the SLM's decision
+    # block on it, and the LLM head with its decision block and the next planning
+    "alg1_plus_b64": ("c4_slm_b64", "c4_llm_b64"),
     # R-Stitch+ step, two launches: SLM head on 64 sequences, then the router on the rows the entropy rule
     # routed with the compaction of its refined mask in the same kernel
     "c4_router": ("c4_slm_b64",),
@@ -372,7 +376,7 @@ def default_steps(workload: str):
     """(steps, warm-up, rotating buffers) when the command line leaves them open."""
     if workload == "c5_catchup":
         return 64, 3, 2
-    if workload in ("c4_batched", "alg1_b64"):
+    if workload in ("c4_batched", "alg1_b64", "alg1_plus_b64"):
         return 2048, 64, 8
     return 8192, 64, 8
 
@@ -419,7 +423,8 @@ def measure(rs, torch, dist, rank, local_rank, world, args, workload: str, K: in
         return None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
 
     stream = torch.cuda.current_stream()
-    alg1 = workload == "alg1_b64"
+    alg1 = workload in ("alg1_b64", "alg1_plus_b64")
+    alg1_plus = workload == "alg1_plus_b64"
     state = None
     if alg1:
         B0 = gen.WORKLOADS[names[0]].B
@@ -428,7 +433,7 @@ def measure(rs, torch, dist, rank, local_rank, world, args, workload: str, K: in
         # fitted coefficients printed in the paper's latency-regression appendix (SLM-1.5B, LLM-7B), ms
         lat_models = [rs.LatencyModel(0.000021, 0.000231, -0.121046, 27.090929),
                       rs.LatencyModel(0.000027, 0.000031, -0.045256, 27.040801)]
-    with_router = workload == "c4_router"
+    with_router = workload == "c4_router" or alg1_plus
     router = None
     if with_router:
         d0 = gen.WORKLOADS[names[0]].d
@@ -463,7 +468,7 @@ def measure(rs, torch, dist, rank, local_rank, world, args, workload: str, K: in
                     alg1_tails.append(state.tail(hi, -1, spans=False, plan_next=(hi == 1), t_max=1 << 30,
                                                  latency=lat_models))
                 kw = dict(R=w.B, B=w.B, n_rows_dev=state.run_count[hi], flags=args.flags, stream=stream,
-                          alg1_tail=alg1_tails[hi])
+                          alg1_tail=None if (alg1_plus and hi == 0) else alg1_tails[hi])
             elif hi == 1:
                 # batched step: the LLM head runs on the subset the SLM head routed, count on device
                 kw.update(row_idx=prev_out[i].llm_idx, n_rows_dev=prev_out[i].llm_count)
@@ -481,11 +486,16 @@ def measure(rs, torch, dist, rank, local_rank, world, args, workload: str, K: in
 
     def step(i):
         calls = prepared[i % n_rot]
-        for call in calls:
+        for ci, call in enumerate(calls):
             st = call.launch()
             if st != 0:
                 raise rs.RstitchError(st, "rstitch_route_ex")
-        if with_router:
+            if alg1_plus and ci == 0:
+                o = call.out
+                router.route(call._keep[1], 64, o.llm_idx, o.mask, r_idx, r_cnt, n_rows_dev=o.llm_count,
+                             logits=r_logits, switch=r_switch, stream=stream, alg1_tail=alg1_tails[0], tok=o.tok,
+                             n_seq_dev=state.run_count[0])
+        if with_router and not alg1_plus:
             o = calls[0].out
             router.route(calls[0]._keep[1], 64, o.llm_idx, o.mask, r_idx, r_cnt, n_rows_dev=o.llm_count,
                          logits=r_logits, switch=r_switch, stream=stream)
@@ -767,7 +777,7 @@ def main() -> int:
         peaks = measured_peaks()
         read = read_stream_ceiling(rs, torch, dev, torch.cuda.current_stream()) if world == 1 else {"gbs": None}
         sec = ms / 1e3
-        w0, alg1 = res["w0"], args.workload == "alg1_b64"
+        w0, alg1 = res["w0"], args.workload in ("alg1_b64", "alg1_plus_b64")
         value = world * res["rows_per_step"] * K / sec
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,

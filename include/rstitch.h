@@ -312,6 +312,8 @@ typedef struct rstitch_router_s {
  *   logits_out  float32 [R, 2];  switch_out optional uint8 [R] (1 = hand the step to the LLM; a tie keeps
  *   the SLM);  refine_mask optional uint8 [n_src] (needs row_idx): refine_mask[row_idx[r]] = switch, which
  *   turns the entropy rule's route_mask into the router's; compact it again with rstitch_compact.
+ * An entry of row_idx outside [0, n_src) reads row 0, gets switch 0 and leaves refine_mask alone; R > 0 with
+ * n_src = 0 is an invalid argument.
  */
 int rstitch_router_forward(const rstitch_router_t *w, const void *hidden, int n_src, const int32_t *row_idx,
                            const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out,
@@ -329,6 +331,26 @@ int rstitch_router_forward(const rstitch_router_t *w, const void *hidden, int n_
 int rstitch_router_route(const rstitch_router_t *w, const void *hidden, int n_src, const int32_t *row_idx,
                          const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out,
                          uint8_t *route_mask, int32_t *llm_idx, int32_t *llm_count, void *cuda_stream);
+
+/*
+ * The SLM's step of an R-Stitch+ round (Algorithm 1: "if H_t > tau: switch <- (argmax_a pi(a | s_t) = LLM);
+ * if active = SLM and switch: discard y_t, roll back, active <- LLM"; Section 3.3: low-entropy tokens
+ * always stay with the SLM).  Issued behind the SLM head's rstitch_route_ex call of the round, which was
+ * made WITHOUT an alg1_tail: rstitch_router_route on that call's llm_idx / llm_count (the run entries
+ * whose entropy exceeded tau) refines its route_mask to (H_t > tau and switch), and the kernel's last block
+ * then runs Algorithm 1's decision block for the SLM's batch on the refined mask and the call's tokens
+ * -- exactly rstitch_alg1_commit(model 0, tok, route_mask) -- and, with plan_next, the next planning.  A
+ * round is then three launches (SLM head, this, LLM head with its own alg1_tail), all on the device.
+ *   n_seq_dev   optional device int32 [1]: the live length of route_mask (the SLM call's n_rows_dev, i.e.
+ *               its run count); entries at or past it are neither compacted nor decided.  NULL: n_src.
+ *   tok         device int32: the SLM call's tok_out;  alg1_tail: as in rstitch_args_t, model must be 0.
+ * The other arguments are those of rstitch_router_route.  Entries of row_idx outside [0, n_src) read row 0,
+ * leave route_mask alone and get switch 0.
+ */
+int rstitch_router_route_alg1(const rstitch_router_t *w, const void *hidden, int n_src, const int32_t *n_seq_dev,
+                              const int32_t *row_idx, const int32_t *n_rows_dev, int R, float *logits_out,
+                              uint8_t *switch_out, uint8_t *route_mask, int32_t *llm_idx, int32_t *llm_count,
+                              const int32_t *tok, const rstitch_alg1_tail_t *alg1_tail, void *cuda_stream);
 
 /* Handle: owns the scratch memory and the device status word for problems up to the given maxima on
  * the current device.  rstitch_destroy(NULL) is a no-op. */

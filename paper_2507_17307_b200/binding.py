@@ -24,6 +24,7 @@ EXPORTS = [
     "rstitch_workspace_bytes", "rstitch_compact", "rstitch_last_status", "rstitch_status_string",
     "rstitch_path_name", "rstitch_route_static", "rstitch_route_ex_host",
     "rstitch_alg1_init", "rstitch_alg1_plan", "rstitch_alg1_commit", "rstitch_router_forward",
+    "rstitch_router_route", "rstitch_router_route_alg1", "rstitch_probe_read_stream",
 ]
 
 
@@ -137,6 +138,9 @@ def lib():
         L.rstitch_router_forward.restype = i
         L.rstitch_router_route.argtypes = [C.POINTER(_Router), vp, i, vp, vp, i, vp, vp, vp, vp, vp, vp]
         L.rstitch_router_route.restype = i
+        L.rstitch_router_route_alg1.argtypes = [C.POINTER(_Router), vp, i, vp, vp, vp, i, vp, vp, vp, vp, vp, vp,
+                                                C.POINTER(_Alg1Tail), vp]
+        L.rstitch_router_route_alg1.restype = i
         L.rstitch_alg1_init.argtypes = [C.POINTER(_Alg1State), i, vp, vp]
         L.rstitch_alg1_init.restype = i
         L.rstitch_alg1_plan.argtypes = [C.POINTER(_Alg1State), i, i, i, C.POINTER(LatencyModel), vp, vp, vp, vp, vp, vp]
@@ -596,14 +600,26 @@ class Router:
         return logits, switch
 
     def route(self, hidden, R: int, row_idx, route_mask, llm_idx, llm_count, n_rows_dev=None, logits=None,
-              switch=None, stream=None, check: bool = True):
+              switch=None, stream=None, check: bool = True, alg1_tail=None, tok=None, n_seq_dev=None):
         """rstitch_router_route: the router on the rows row_idx names, route_mask refined in place and
-        compacted into llm_idx / llm_count by the same launch; returns (logits, switch)."""
+        compacted into llm_idx / llm_count by the same launch; returns (logits, switch).  With alg1_tail
+        (and tok, the SLM call's tokens) it is rstitch_router_route_alg1: the launch goes on with
+        Algorithm 1's decision block for the SLM's batch on the refined mask."""
         import torch
         if logits is None:
             logits = torch.zeros((max(R, 1), 2), dtype=torch.float32, device=hidden.device)
         if switch is None:
             switch = torch.full((max(R, 1),), 255, dtype=torch.uint8, device=hidden.device)
+        if alg1_tail is not None:
+            st = lib().rstitch_router_route_alg1(C.byref(self._c), _ptr(hidden), int(hidden.shape[0]), _ptr(n_seq_dev),
+                                                 _ptr(row_idx), _ptr(n_rows_dev), int(R), _ptr(logits), _ptr(switch),
+                                                 _ptr(route_mask), _ptr(llm_idx), _ptr(llm_count), _ptr(tok),
+                                                 C.byref(alg1_tail), _stream_ptr(stream))
+            if not check:
+                return st
+            if st != 0:
+                raise RstitchError(st, "rstitch_router_route_alg1")
+            return logits, switch
         st = lib().rstitch_router_route(C.byref(self._c), _ptr(hidden), int(hidden.shape[0]), _ptr(row_idx),
                                         _ptr(n_rows_dev), int(R), _ptr(logits), _ptr(switch), _ptr(route_mask),
                                         _ptr(llm_idx), _ptr(llm_count), _stream_ptr(stream))

@@ -29,6 +29,38 @@ struct rstitch_handle_s {
     unsigned launch_count = 0;           // kernels enqueued since the status word was last read
 };
 
+namespace rstitch {
+
+// rstitch_alg1_tail_t (host) -> the device copy the tails carry; false: a bad structure.
+bool make_alg1_tail(const rstitch_alg1_tail_t *t, Alg1Tail *out)
+{
+    out->on = 0;
+    if (!t) return true;
+    if (!alg1_state_ok(t->state) || t->n_seq < 0 || (t->model != 0 && t->model != 1) || !t->run_count ||
+        (t->n_seq > 0 && !t->run_idx))
+        return false;
+    out->on = 1;
+    out->s = *t->state;
+    out->n_seq = t->n_seq; out->model = t->model;
+    out->run_idx = t->run_idx; out->run_count = t->run_count; out->row_off = t->row_off;
+    out->eos_id = t->eos_id; out->plan_next = t->plan_next ? 1 : 0; out->t_max = t->t_max;
+    for (int m = 0; m < 2; ++m) {
+        out->lat[m] = t->latency[m];
+        out->nx_idx[m] = t->next_run_idx[m]; out->nx_cnt[m] = t->next_run_count[m];
+        out->nx_ninf[m] = t->next_n_inf[m]; out->nx_nkv[m] = t->next_n_kv[m]; out->nx_off[m] = t->next_row_off[m];
+        if (t->plan_next) {
+            if (t->t_max < 0 || !out->nx_cnt[m] || !out->nx_off[m]) return false;
+            if (t->n_seq > 0 && (!out->nx_idx[m] || !out->nx_ninf[m] || !out->nx_nkv[m])) return false;
+            if (!std::isfinite(t->latency[m].a) || !std::isfinite(t->latency[m].b) ||
+                !std::isfinite(t->latency[m].c) || !std::isfinite(t->latency[m].d))
+                return false;
+        }
+    }
+    return true;
+}
+
+}  // namespace rstitch
+
 namespace {
 
 constexpr size_t kMirrorMax = 16 * 1024;        // host-buffer calls: outputs up to this size are written to the host by the kernel
@@ -189,34 +221,6 @@ bool use_umma(int R, int d, int V, uint32_t flags)
     if (!umma_shape_ok(R, d, V)) return false;       // tiny shapes stay on the streaming kernel
     if (flags & RSTITCH_PATH_UMMA) return true;
     return R > kGemvMaxRows;
-}
-
-// rstitch_alg1_tail_t (host) -> the device copy the tails carry; false: a bad structure.
-bool make_alg1_tail(const rstitch_alg1_tail_t *t, Alg1Tail *out)
-{
-    out->on = 0;
-    if (!t) return true;
-    if (!alg1_state_ok(t->state) || t->n_seq < 0 || (t->model != 0 && t->model != 1) || !t->run_count ||
-        (t->n_seq > 0 && !t->run_idx))
-        return false;
-    out->on = 1;
-    out->s = *t->state;
-    out->n_seq = t->n_seq; out->model = t->model;
-    out->run_idx = t->run_idx; out->run_count = t->run_count; out->row_off = t->row_off;
-    out->eos_id = t->eos_id; out->plan_next = t->plan_next ? 1 : 0; out->t_max = t->t_max;
-    for (int m = 0; m < 2; ++m) {
-        out->lat[m] = t->latency[m];
-        out->nx_idx[m] = t->next_run_idx[m]; out->nx_cnt[m] = t->next_run_count[m];
-        out->nx_ninf[m] = t->next_n_inf[m]; out->nx_nkv[m] = t->next_n_kv[m]; out->nx_off[m] = t->next_row_off[m];
-        if (t->plan_next) {
-            if (t->t_max < 0 || !out->nx_cnt[m] || !out->nx_off[m]) return false;
-            if (t->n_seq > 0 && (!out->nx_idx[m] || !out->nx_ninf[m] || !out->nx_nkv[m])) return false;
-            if (!std::isfinite(t->latency[m].a) || !std::isfinite(t->latency[m].b) ||
-                !std::isfinite(t->latency[m].c) || !std::isfinite(t->latency[m].d))
-                return false;
-        }
-    }
-    return true;
 }
 
 // Validated arguments -> kernels.  With shard_stats the head is a vocabulary shard starting at entry

@@ -60,6 +60,7 @@ cudaError_t launch_shard_merge(const float *gathered, int n_shards, const int32_
 // Algorithm 1's block after a routing call that has no rows of its own (one small launch), and the
 // check of a caller's state structure.
 bool        alg1_state_ok(const rstitch_alg1_state_t *s);
+bool        make_alg1_tail(const rstitch_alg1_tail_t *t, Alg1Tail *out);   // host structure -> what the kernels carry; false: bad
 cudaError_t launch_alg1_tail(const Alg1Tail &a, const int32_t *tok, const uint8_t *mask, cudaStream_t stream);
 
 // The bounded wait running out on purpose (rstitch_selftest_wait): site id it leaves in the status word.

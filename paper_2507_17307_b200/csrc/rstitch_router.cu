@@ -118,7 +118,8 @@ __device__ __forceinline__ void router_row(const rstitch_router_t &w, const unsi
 {
     float *s = sm, *x = sm + w.d, *t = x + w.h;
     int src = row_idx ? row_idx[r] : r;
-    if (src < 0 || src >= n_src) src = 0;
+    const bool valid = src >= 0 && src < n_src;      // an entry outside [0, n_src) reads row 0 and decides nothing
+    if (!valid) src = 0;
     const unsigned short *hrow = hidden + (size_t)src * w.d;
     for (int k = threadIdx.x; k < w.d; k += kThreads) s[k] = __uint_as_float((unsigned)hrow[k] << 16);
     float *blk = t + w.ff;                        // staged block weights
@@ -279,11 +280,11 @@ __device__ __forceinline__ void router_row(const rstitch_router_t &w, const unsi
         a0 = warp_sum(a0) + p_b_out[0];
         a1 = warp_sum(a1) + p_b_out[1];
         if (lane == 0) {
-            const uint8_t sw = a1 > a0 ? 1 : 0;                     // a tie keeps the SLM
+            const uint8_t sw = (valid && a1 > a0) ? 1 : 0;          // a tie keeps the SLM
             logits_out[2 * r] = a0;
             logits_out[2 * r + 1] = a1;
             if (switch_out) switch_out[r] = sw;
-            if (refine_mask && row_idx) refine_mask[src] = sw;
+            if (refine_mask && row_idx && valid) refine_mask[src] = sw;
         }
     }
 }
@@ -296,7 +297,8 @@ __device__ unsigned g_router_ticket = 0;
 __global__ void __launch_bounds__(kThreads, 1)
 router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const int32_t *row_idx,
               const int32_t *n_rows_dev, int R, float *logits_out, uint8_t *switch_out, uint8_t *refine_mask,
-              int stage_weights, int32_t *cmp_idx, int32_t *cmp_count)
+              int stage_weights, int32_t *cmp_idx, int32_t *cmp_count, const int32_t *n_seq_dev, const int32_t *tok,
+              rstitch::Alg1Tail alg1)
 {
     extern __shared__ __align__(16) float sm[];   // [d] hidden row | [h] x | [ff] t | [ff h] W1 | [h ff] W2 of a block
     __shared__ int s_tail[66];
@@ -312,7 +314,11 @@ router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    rstitch::tail_compact(refine_mask, n_src, nullptr, nullptr, cmp_idx, cmp_count, nullptr, nullptr, nullptr, s_tail);
+    int n_seq = n_src;                              // mask entries that are live in this round
+    if (n_seq_dev) { int n = *n_seq_dev; n_seq = n < 0 ? 0 : (n < n_src ? n : n_src); }
+    rstitch::tail_compact(refine_mask, n_seq, nullptr, nullptr, cmp_idx, cmp_count, nullptr, nullptr, nullptr, s_tail);
+    // Algorithm 1, R-Stitch+ lines: the SLM's decision block runs on the mask the router has just refined
+    if (alg1.on) rstitch::alg1_tail_block(alg1, tok, refine_mask, s_tail);
     if (threadIdx.x == 0) g_router_ticket = 0u;
 }
 
@@ -321,9 +327,12 @@ router_kernel(rstitch_router_t w, const unsigned short *hidden, int n_src, const
 static int router_launch(const rstitch_router_t *w, const void *hidden, int n_src,
                          const int32_t *row_idx, const int32_t *n_rows_dev, int R,
                          float *logits_out, uint8_t *switch_out, uint8_t *refine_mask,
-                         int32_t *cmp_idx, int32_t *cmp_count, void *cuda_stream)
+                         int32_t *cmp_idx, int32_t *cmp_count, void *cuda_stream,
+                         const int32_t *n_seq_dev = nullptr, const int32_t *tok = nullptr,
+                         const rstitch::Alg1Tail *alg1 = nullptr)
 {
     if (!w || R < 0 || n_src < 0 || !logits_out) return RSTITCH_ERR_INVALID_ARG;
+    if (R > 0 && n_src == 0) return RSTITCH_ERR_INVALID_ARG;           // rows to read, but none present
     if (w->d < 1 || w->h < 1 || w->ff < 1 || w->n_blocks < 0) return RSTITCH_ERR_INVALID_ARG;
     if (w->h > kMaxH || w->ff > kMaxFF || w->d > 16384) return RSTITCH_ERR_UNSUPPORTED_SHAPE;
     if (!w->W_in || !w->b_in || !w->ln_g || !w->ln_b || !w->W_out || !w->b_out) return RSTITCH_ERR_INVALID_ARG;
@@ -357,7 +366,8 @@ static int router_launch(const rstitch_router_t *w, const void *hidden, int n_sr
     }
     router_kernel<<<R, kThreads, smem, (cudaStream_t)cuda_stream>>>(*w, (const unsigned short *)hidden, n_src, row_idx,
                                                                     n_rows_dev, R, logits_out, switch_out, refine_mask,
-                                                                    stage_weights, cmp_idx, cmp_count);
+                                                                    stage_weights, cmp_idx, cmp_count, n_seq_dev, tok,
+                                                                    alg1 ? *alg1 : rstitch::Alg1Tail{});
     if (cudaGetLastError() != cudaSuccess) return RSTITCH_ERR_CUDA;
     return RSTITCH_OK;
 }
@@ -381,4 +391,29 @@ extern "C" int rstitch_router_route(const rstitch_router_t *w, const void *hidde
     if (R == 0) return rstitch_compact(route_mask, n_src, llm_idx, llm_count, cuda_stream);
     return router_launch(w, hidden, n_src, row_idx, n_rows_dev, R, logits_out, switch_out, route_mask, llm_idx,
                          llm_count, cuda_stream);
+}
+
+extern "C" int rstitch_router_route_alg1(const rstitch_router_t *w, const void *hidden, int n_src,
+                                         const int32_t *n_seq_dev, const int32_t *row_idx, const int32_t *n_rows_dev,
+                                         int R, float *logits_out, uint8_t *switch_out, uint8_t *route_mask,
+                                         int32_t *llm_idx, int32_t *llm_count, const int32_t *tok,
+                                         const rstitch_alg1_tail_t *alg1_tail, void *cuda_stream)
+{
+    if (!row_idx || !route_mask || !llm_count || (n_src > 0 && !llm_idx) || !alg1_tail || !tok)
+        return RSTITCH_ERR_INVALID_ARG;
+    if (n_src > 65536) return RSTITCH_ERR_UNSUPPORTED_SHAPE;             // one block compacts the mask
+    rstitch::Alg1Tail alg1;
+    if (!rstitch::make_alg1_tail(alg1_tail, &alg1) || alg1.model != 0) return RSTITCH_ERR_INVALID_ARG;
+    if (R == 0 || n_src == 0) {
+        // no row can have crossed the threshold: the compaction of the mask as it stands, then the block
+        int st = rstitch_compact(route_mask, n_src, llm_idx, llm_count, cuda_stream);
+        if (st != RSTITCH_OK) return st;
+        if (rstitch::launch_alg1_tail(alg1, tok, route_mask, (cudaStream_t)cuda_stream) != cudaSuccess) {
+            cudaGetLastError();
+            return RSTITCH_ERR_CUDA;
+        }
+        return RSTITCH_OK;
+    }
+    return router_launch(w, hidden, n_src, row_idx, n_rows_dev, R, logits_out, switch_out, route_mask, llm_idx,
+                         llm_count, cuda_stream, n_seq_dev, tok, &alg1);
 }

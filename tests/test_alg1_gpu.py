@@ -314,3 +314,133 @@ def test_fused_loop_replays_from_one_cuda_graph(rs, oracle):
     for h in handles:
         assert rs.last_status(h)["timeouts"] == 0
         h.destroy()
+
+
+def test_rstitch_plus_rounds_with_the_router_in_the_loop(rs, oracle):
+    # Algorithm 1 with its R-Stitch+ lines, batched and on the device: a round is the SLM head's call
+    # (no decision block of its own), the router on the rows whose entropy exceeded tau -- its last block
+    # refines the mask to (H > tau and switch), compacts it and runs the SLM's decision block on it --
+    # and the LLM head's call with its decision block and the next planning.  Three launches, no host
+    # work; the rounds are issued directly and replayed from one CUDA graph, and the final state is the
+    # oracle's per-sequence loop fed the oracle router's switches.
+    import torch
+    B, rounds, tau, eos = 48, 7, 0.3, -1
+    c = coeffs()
+    lat = [rs.LatencyModel(*c["SLM-1.5B"]), rs.LatencyModel(*c["LLM-7B"])]
+    for seed in range(40):
+        ws = [gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=256, V=2053, seed=8600 + seed, diffuse_frac=(0.6, 0.6)),
+              gen.scaled(gen.WORKLOADS["c4_llm_b64"], B=B, d=320, V=3001, seed=8700 + seed, diffuse_frac=(0.6, 0.6))]
+        w_bits = [gen.make_w_head(w) for w in ws]
+        pools_bits = [gen.make_hidden(ws[m], w_bits[m], 0)[0] for m in (0, 1)]
+        refs = [oracle.route(pools_bits[m], w_bits[m], tau) for m in (0, 1)]
+        rw = gen.make_router_weights(256, 32, 64, 6, seed=900 + seed)
+        r_logits, r_sw = oracle.router_rows(pools_bits[0], rw)
+        clear = all((np.abs(r["ent"] - tau) > 4 * ENT_TOL).all() and (r["gap"] > GAP_TOL).all() for r in refs)
+        unsure = refs[0]["ent"] > tau
+        if clear and (np.abs(r_logits[:, 1] - r_logits[:, 0]) > 1e-3).all() and \
+                0 < r_sw[unsure].sum() < unsure.sum():          # the router keeps some rows and hands some over
+            break
+    else:
+        raise AssertionError("no seed kept every row clear of the tolerance bands")
+    w_dev = [to_dev_bf16(b) for b in w_bits]
+    pools = [to_dev_bf16(p) for p in pools_bits]
+    router = rs.Router({k: torch.from_numpy(v).cuda() for k, v in rw.items()})
+    prompt = to_dev_i32(np.arange(3, 3 + B))
+    handles = [rs.Handle(64, 256, 4096), rs.Handle(64, 320, 4096)]
+    side = torch.cuda.Stream()
+
+    def make(state):
+        tails = [state.tail(0, eos, spans=False), state.tail(1, eos, spans=False, plan_next=True, t_max=rounds, latency=lat)]
+        outs = [rs.RouteOutputs.allocate(B, B, "cuda") for _ in (0, 1)]
+        slm = rs.PreparedCall(handles[0], pools[0], w_dev[0], tau, outs[0], n_rows_dev=state.run_count[0], stream=side)
+        llm = rs.PreparedCall(handles[1], pools[1], w_dev[1], tau, outs[1], n_rows_dev=state.run_count[1], stream=side,
+                              alg1_tail=tails[1])
+        bufs = {"logits": torch.zeros((B, 2), dtype=torch.float32, device="cuda"),
+                "switch": torch.zeros(B, dtype=torch.uint8, device="cuda"),
+                "idx": torch.full((B,), -1, dtype=torch.int32, device="cuda"),
+                "cnt": torch.full((1,), -1, dtype=torch.int32, device="cuda")}
+
+        def one_round():
+            assert slm.launch() == 0
+            router.route(pools[0], B, outs[0].llm_idx, outs[0].mask, bufs["idx"], bufs["cnt"],
+                         n_rows_dev=outs[0].llm_count, logits=bufs["logits"], switch=bufs["switch"], stream=side,
+                         alg1_tail=tails[0], tok=outs[0].tok, n_seq_dev=state.run_count[0])
+            assert llm.launch() == 0
+        return one_round, (tails, outs, slm, llm, bufs)
+
+    def start(state):
+        with torch.cuda.stream(side):
+            state.init(prompt, stream=side)
+            state.plan(0, rounds, lat[0], stream=side)
+            state.plan(1, rounds, lat[1], stream=side)
+
+    direct, graphed = rs.Alg1State(B, y_cap=rounds), rs.Alg1State(B, y_cap=rounds)
+    round_d, keep_d = make(direct)
+    start(direct)
+    with torch.cuda.stream(side):
+        for _ in range(rounds):
+            round_d()
+    side.synchronize()
+    round_g, keep_g = make(graphed)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        for _ in range(rounds):
+            round_g()
+    start(graphed)
+    side.synchronize()
+    g.replay()
+    torch.cuda.synchronize()
+    a, b = state_to_host(direct), state_to_host(graphed)
+    for k in a:
+        assert np.array_equal(a[k], b[k]), k
+    # the oracle's loop per sequence, fed what each sequence saw: as run entry j of a model's batch it
+    # read row j of that model's pool, and on the SLM the router's switch for that row
+    active = np.zeros(B, dtype=np.int64)
+    tok_s = np.zeros((2, B, rounds), dtype=np.int32)
+    ent_s = np.zeros((2, B, rounds))
+    sw_s = np.zeros((B, rounds), dtype=np.uint8)
+    kept_on_slm_despite_entropy = 0
+    for t in range(rounds):
+        nxt = active.copy()
+        for m in (0, 1):
+            for j, sid in enumerate(np.flatnonzero(active == m)):
+                tok_s[m, sid, t], ent_s[m, sid, t] = refs[m]["tok"][j], refs[m]["ent"][j]
+                unsure_j = refs[m]["ent"][j] > tau
+                if m == 0:
+                    sw_s[sid, t] = r_sw[j]
+                    nxt[sid] = 1 if (unsure_j and r_sw[j]) else 0
+                    kept_on_slm_despite_entropy += int(unsure_j and not r_sw[j])
+                else:
+                    nxt[sid] = 1 if unsure_j else 0
+        active = nxt
+    assert kept_on_slm_despite_entropy > 0, "the router never overruled the entropy rule"
+    differs = 0
+    for sid in range(B):
+        ref = oracle.alg1_sequence(3 + sid, rounds, tau, eos, tok_s[0, sid], ent_s[0, sid], tok_s[1, sid], ent_s[1, sid],
+                                   c["SLM-1.5B"], c["LLM-7B"], switch_slm=sw_s[sid])
+        check_against_oracle(oracle, a, sid, ref)
+        plain = oracle.alg1_sequence(3 + sid, rounds, tau, eos, tok_s[0, sid], ent_s[0, sid], tok_s[1, sid],
+                                     ent_s[1, sid], c["SLM-1.5B"], c["LLM-7B"])
+        differs += int(plain["y"].tolist() != ref["y"].tolist() or plain["active"] != ref["active"])
+    assert differs > 0, "R-Stitch+ and R-Stitch gave the same trajectories: the test would not tell them apart"
+    assert a["kept"][1].sum() > 0 and a["kept"][0].sum() > 0
+    for h in handles:
+        assert rs.last_status(h)["timeouts"] == 0
+        h.destroy()
+
+
+def test_router_route_alg1_argument_errors(rs):
+    import torch
+    rw = gen.make_router_weights(64, 16, 32, 2, seed=5)
+    router = rs.Router({k: torch.from_numpy(v).cuda() for k, v in rw.items()})
+    st = rs.Alg1State(8, y_cap=4)
+    hid = torch.zeros((8, 64), dtype=torch.bfloat16, device="cuda")
+    idx = torch.zeros(8, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    mask = torch.zeros(8, dtype=torch.uint8, device="cuda")
+    tok = torch.zeros(8, dtype=torch.int32, device="cuda")
+    tail = st.tail(1, -1, spans=False)                       # the LLM's block has no business here
+    assert router.route(hid, 8, idx, mask, idx.clone(), cnt, alg1_tail=tail, tok=tok, check=False) == -1
+    tail = st.tail(0, -1, spans=False)
+    assert router.route(hid, 8, idx, mask, idx.clone(), cnt, alg1_tail=tail, tok=None, check=False) == -1
+    torch.cuda.synchronize()
