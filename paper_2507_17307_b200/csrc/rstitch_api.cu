@@ -27,6 +27,7 @@ struct rstitch_handle_s {
     void    *st_in = nullptr;  size_t st_in_bytes = 0;       // pinned mirror of its input part (small inputs)
     cudaStream_t last_stream = nullptr;
     unsigned launch_count = 0;           // kernels enqueued since the status word was last read
+    TmapCache tmaps;                     // encoded tensor maps of the tensor-core kernels
 };
 
 namespace rstitch {
@@ -287,7 +288,7 @@ int enqueue_head(rstitch_handle_s *h, const rstitch_args_t *a, cudaStream_t stre
         // the partials region is sized for the shape the scratch was made for
         size_t part = a->workspace ? ws_partials_bytes(a->R, a->V) : ws_partials_bytes(h->maxR, h->maxV);
         e = launch_head_umma(ha, ta, sc, (char *)ws + kWsHeader + part, h->sm_count, stream, &launched,
-                             (a->flags & RSTITCH_PATH_PAIR) != 0);
+                             (a->flags & RSTITCH_PATH_PAIR) != 0, &h->tmaps);
     } else {
         e = launch_head_gemv(ha, ta, sc, h->sm_count, stream, &launched);
     }

@@ -41,10 +41,22 @@ cudaError_t launch_head_gemv(const HeadArgs &h, const TailArgs &t, const Scratch
 
 // Tensor-core kernel (tcgen05 + tensor memory): any row count; the choice between the two is the
 // caller's.  gather_buf (umma_gather_bytes(R, d) bytes, 256-byte aligned) is used only with row_idx.
+// Encoded tensor maps by (base pointer, rows, d, box rows), least recently used replaced; owned by a
+// handle and touched only on the host, by the thread that enqueues through that handle.
+struct TmapCache {
+    struct Entry {
+        const void *base = nullptr;
+        int rows = 0, d = 0, box_rows = 0;
+        unsigned long long used = 0;             // 0: empty
+        alignas(64) unsigned char map[128];
+    } e[24];
+    unsigned long long clock = 0;
+};
 bool        umma_shape_ok(int R, int d, int V);
 size_t      umma_gather_bytes(int R, int d);
 cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
-                             int sm_count, cudaStream_t stream, int *launched, bool use_pair);
+                             int sm_count, cudaStream_t stream, int *launched, bool use_pair,
+                             TmapCache *cache = nullptr);
 
 // The cross-block merge and the routing tail as a launch of its own, behind a head kernel that was
 // launched without its fused tail (rstitch_finalize.cu).  Both launches carry the programmatic stream

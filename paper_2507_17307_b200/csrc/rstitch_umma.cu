@@ -24,6 +24,7 @@
 #include "rstitch_ptx.cuh"
 
 #include <cuda.h>
+#include <cstring>
 
 namespace rstitch {
 
@@ -970,7 +971,7 @@ EncodeTiledFn encode_fn()
 
 // bf16 [rows, d] row-major, box = 64 elements along d by box_rows rows, 128-byte swizzle,
 // out-of-range elements read as zero.
-bool make_map(CUtensorMap *m, const void *base, int rows, int d, int box_rows)
+bool encode_map(CUtensorMap *m, const void *base, int rows, int d, int box_rows)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
@@ -981,6 +982,27 @@ bool make_map(CUtensorMap *m, const void *base, int rows, int d, int box_rows)
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The same through the caller's cache: a decode loop presents the same W_head and the same hidden
+// buffers call after call, and encoding six maps costs the host more than the two launches do.
+bool make_map(TmapCache *cache, CUtensorMap *m, const void *base, int rows, int d, int box_rows)
+{
+    if (!cache) return encode_map(m, base, rows, d, box_rows);
+    TmapCache::Entry *victim = &cache->e[0];
+    for (TmapCache::Entry &e : cache->e) {
+        if (e.used && e.base == base && e.rows == rows && e.d == d && e.box_rows == box_rows) {
+            e.used = ++cache->clock;
+            std::memcpy(m, e.map, sizeof(CUtensorMap));
+            return true;
+        }
+        if (e.used < victim->used) victim = &e;
+    }
+    if (!encode_map(m, base, rows, d, box_rows)) return false;
+    victim->base = base; victim->rows = rows; victim->d = d; victim->box_rows = box_rows;
+    victim->used = ++cache->clock;
+    std::memcpy(victim->map, m, sizeof(CUtensorMap));
+    return true;
 }
 
 }  // namespace
@@ -996,8 +1018,10 @@ size_t umma_gather_bytes(int R, int d)
     return rows * (size_t)d * 2;
 }
 
+static_assert(sizeof(CUtensorMap) == sizeof(TmapCache::Entry::map), "tensor-map cache entry size");
+
 cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
-                             int sm_count, cudaStream_t stream, int *launched, bool use_pair)
+                             int sm_count, cudaStream_t stream, int *launched, bool use_pair, TmapCache *cache)
 {
     *launched = 0;
     static bool configured[64] = {};
@@ -1054,9 +1078,9 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
     }
     CUtensorMap tm_h;
     WMaps tm_w;
-    if (!make_map(&tm_h, hid_base, hid_rows, h.d, plan.a_rows)) return cudaErrorInvalidValue;
+    if (!make_map(cache, &tm_h, hid_base, hid_rows, h.d, plan.a_rows)) return cudaErrorInvalidValue;
     for (int b = 0; b < 5; ++b)
-        if (!make_map(&tm_w.box[b], h.W, h.V, h.d, 16 << b)) return cudaErrorInvalidValue;
+        if (!make_map(cache, &tm_w.box[b], h.W, h.V, h.d, 16 << b)) return cudaErrorInvalidValue;
     Partials Pk = P;
     HeadArgs hk2 = hk;
     TailArgs tk = t;
