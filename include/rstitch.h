@@ -59,7 +59,6 @@ extern "C" {
 #define RSTITCH_SAMPLE           0x2u  /* tok_out is sampled from softmax(z / temperature), not the greedy token */
 #define RSTITCH_PATH_GEMV        0x10u /* testing only: force the CUDA-core streaming kernel */
 #define RSTITCH_PATH_UMMA        0x20u /* testing only: force the tcgen05 tensor-core kernel */
-#define RSTITCH_PATH_PAIR        0x40u /* testing only: more than 128 rows on pairs of blocks (tcgen05 cta_group::2) */
 
 typedef struct rstitch_handle_s *rstitch_handle_t;
 

@@ -6,5 +6,5 @@ The Python layer only marshals arguments: every step of the path runs in the ker
 from .binding import (  # noqa: F401
     RstitchError, Handle, Alg1State, LatencyModel, Router, RouteOutputs, PreparedCall, PreparedHostCall, route_ex_host, lib, library_path, route, route_ex, route_host, route_static, STATIC_MAX_ROWS, compact, shard_stats, shard_route, SHARD_WORDS, selftest_wait, probe_read_stream, SELFTEST_SITE,
     last_status, workspace_bytes, status_string, path_name,
-    TAU_NORMALIZED, SAMPLE, PATH_GEMV, PATH_UMMA, PATH_PAIR,
+    TAU_NORMALIZED, SAMPLE, PATH_GEMV, PATH_UMMA,
 )

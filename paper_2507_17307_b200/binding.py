@@ -17,7 +17,6 @@ TAU_NORMALIZED = 0x1
 SAMPLE = 0x2
 PATH_GEMV = 0x10
 PATH_UMMA = 0x20
-PATH_PAIR = 0x40
 
 EXPORTS = [
     "rstitch_route", "rstitch_route_ex", "rstitch_route_host", "rstitch_create", "rstitch_destroy",

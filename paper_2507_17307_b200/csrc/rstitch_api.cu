@@ -147,8 +147,7 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a, ValidateMode mo
         if (st != RSTITCH_OK) return st;
         if (a->n_src < 0) return RSTITCH_ERR_INVALID_ARG;
         if ((a->flags & RSTITCH_PATH_GEMV) && (a->flags & RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
-        if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA |
-                         RSTITCH_PATH_PAIR))
+        if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA))
             return RSTITCH_ERR_INVALID_ARG;
         if ((a->flags & RSTITCH_SAMPLE) && !(std::isfinite(a->temperature) && a->temperature > 0.f))
             return RSTITCH_ERR_INVALID_ARG;
@@ -167,8 +166,7 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a, ValidateMode mo
         if (a->R < 0 || a->B < 0 || a->V < 2) return RSTITCH_ERR_INVALID_ARG;
         if (a->R > kMaxRows) return RSTITCH_ERR_UNSUPPORTED_SHAPE;
         if (!std::isfinite(a->tau)) return RSTITCH_ERR_INVALID_ARG;
-        if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA |
-                         RSTITCH_PATH_PAIR))
+        if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA))
             return RSTITCH_ERR_INVALID_ARG;
         if (!a->llm_count) return RSTITCH_ERR_INVALID_ARG;
         if (a->row_seq == nullptr && a->B != a->R) return RSTITCH_ERR_INVALID_ARG;
@@ -189,8 +187,7 @@ int validate(const rstitch_handle_s *h, const rstitch_args_t *a, ValidateMode mo
     if (a->B < 0 || a->n_src < 0) return RSTITCH_ERR_INVALID_ARG;
     if (!std::isfinite(a->tau)) return RSTITCH_ERR_INVALID_ARG;
     if ((a->flags & RSTITCH_PATH_GEMV) && (a->flags & RSTITCH_PATH_UMMA)) return RSTITCH_ERR_INVALID_ARG;
-    if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA |
-                     RSTITCH_PATH_PAIR))
+    if (a->flags & ~(RSTITCH_TAU_NORMALIZED | RSTITCH_SAMPLE | RSTITCH_PATH_GEMV | RSTITCH_PATH_UMMA))
         return RSTITCH_ERR_INVALID_ARG;
     if ((a->flags & RSTITCH_SAMPLE) && !(std::isfinite(a->temperature) && a->temperature > 0.f))
         return RSTITCH_ERR_INVALID_ARG;
@@ -288,7 +285,7 @@ int enqueue_head(rstitch_handle_s *h, const rstitch_args_t *a, cudaStream_t stre
         // the partials region is sized for the shape the scratch was made for
         size_t part = a->workspace ? ws_partials_bytes(a->R, a->V) : ws_partials_bytes(h->maxR, h->maxV);
         e = launch_head_umma(ha, ta, sc, (char *)ws + kWsHeader + part, h->sm_count, stream, &launched,
-                             (a->flags & RSTITCH_PATH_PAIR) != 0, &h->tmaps);
+                             &h->tmaps);
     } else {
         e = launch_head_gemv(ha, ta, sc, h->sm_count, stream, &launched);
     }

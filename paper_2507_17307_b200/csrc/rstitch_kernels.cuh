@@ -55,8 +55,7 @@ struct TmapCache {
 bool        umma_shape_ok(int R, int d, int V);
 size_t      umma_gather_bytes(int R, int d);
 cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
-                             int sm_count, cudaStream_t stream, int *launched, bool use_pair,
-                             TmapCache *cache = nullptr);
+                             int sm_count, cudaStream_t stream, int *launched, TmapCache *cache = nullptr);
 
 // The cross-block merge and the routing tail as a launch of its own, behind a head kernel that was
 // launched without its fused tail (rstitch_finalize.cu).  Both launches carry the programmatic stream

@@ -101,7 +101,7 @@ extern "C" int rstitch_route_static(const void *hidden, const void *W_head, int 
     cudaError_t e;
     if (B > 1 && umma_shape_ok(B, d, V)) {
         int launched = 0;
-        e = launch_head_umma(ha, ta, sc, nullptr, sms, stream, &launched, false);
+        e = launch_head_umma(ha, ta, sc, nullptr, sms, stream, &launched);
     } else {
         e = launch_head_gemv(ha, ta, sc, sms, stream);
     }

@@ -705,225 +705,6 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
     }
 }
 
-// ---- several M tiles, a pair of blocks per W tile (tcgen05 cta_group::2) ---------------------------
-// Measurements of the kernel above put its limit in shared memory: per k-step a block takes 64 KB of TMA
-// writes and 96 KB of MMA operand reads (A 4 KB + B 8 KB per instruction), about what shared memory
-// moves in the time.  Two blocks of a cluster working as a pair halve the B traffic: one instruction
-// computes M = 256 (each block's own 128-row A tile into its own tensor memory) against a 256-row W tile
-// whose rows are split between the two blocks' shared memory, so each block loads and reads only 128 W
-// rows.  Each block still holds two accumulators (two M tiles), i.e. a pair covers four M tiles per W
-// tile.  As it stands this variant wins only where the rows fill whole groups of four M tiles and its
-// coarser work split balances (it lost at 576 rows), so it is opt-in (RSTITCH_PATH_PAIR).
-//   leader (cluster rank 0): its MMA thread issues for the pair; "full" barriers live here and collect
-//     the copy bytes of both blocks; "accumulator empty" collects the arrivals of both blocks' epilogues.
-//   both blocks: producers (own A tiles, own half of W, signalling the leader's barrier), eight epilogue
-//     warps (own rows), "empty" and "accumulator full" barriers fed by multicast tcgen05.commit.
-// Work: cluster c takes vocabulary tiles c, c + #clusters, ...; for each, the groups of four M tiles.
-constexpr int kThreadsP    = 320 + (kProducers - 1) * 32;
-constexpr int kStagesP     = 4;
-constexpr int kStagePBytes = 2 * kABytes + kBBytes / 2;    // 48 KB: two hidden tiles + half a W tile
-constexpr int kDynSmemP    = kStagesP * kStagePBytes + 1024;
-
-__global__ void __launch_bounds__(kThreadsP, 1)
-head_umma_pair_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_constant__ WMaps tm_w,
-                      HeadArgs h, TailArgs t, Partials P, int nM, int n_slices)
-{
-    extern __shared__ unsigned char dyn_smem_raw[];
-    __shared__ __align__(8) uint64_t s_full[kStagesP], s_empty[kStagesP];
-    __shared__ __align__(8) uint64_t s_acc_full, s_acc_empty, s_done;
-    __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort, s_zero;
-
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t rank = ptx::cluster_ctarank();            // 0 = leader
-    const uint32_t ring = (ptx::smem_u32(dyn_smem_raw) + 1023u) & ~1023u;
-    const int nK = (h.d + kTileK - 1) / kTileK;
-    ptx::grid_dep_launch_dependents();
-    ptx::grid_dep_wait();          // hidden rows, the live count and the scratch may come from the kernels before
-    int R_live = h.R;
-    if (h.n_rows_dev) { int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
-    const int nG = (nM + 3) / 4;                             // groups of four M tiles
-    const int nVT = (h.V + kTileNMax - 1) / kTileNMax;
-    const int cluster = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
-    const int n_vt = (cluster < nVT && R_live > 0) ? (nVT - cluster + n_clusters - 1) / n_clusters : 0;
-    const int n_items = n_vt * nG;
-
-    if (threadIdx.x == 0) {
-        s_abort = 0; s_zero = 0;
-        for (int s = 0; s < kStagesP; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&s_full[s]), 1);     // the leader's producer arrives, both blocks' bytes
-            ptx::mbar_init(ptx::smem_u32(&s_empty[s]), 1);    // one multicast commit
-        }
-        ptx::mbar_init(ptx::smem_u32(&s_acc_full), 1);
-        ptx::mbar_init(ptx::smem_u32(&s_acc_empty), 16);      // eight epilogue warps in each block
-        ptx::mbar_init(ptx::smem_u32(&s_done), 1);
-        ptx::mbar_fence_init();
-        ptx::prefetch_tmap(&tm_hidden);
-        ptx::prefetch_tmap(&tm_w.box[3]);
-    }
-    if (warp == 1) {
-        ptx::tmem_alloc_pair(ptx::smem_u32(&s_tmem_base), kTmemCols);
-        ptx::tmem_relinquish_pair();
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    ptx::cluster_sync();               // the peer's barriers and tensor memory exist from here on
-    ptx::tc_fence_after_sync();
-    const uint32_t tmem_base = s_tmem_base;
-
-    if (warp == 0 || warp >= 10) {
-        // ---- producers (both blocks): the copies of a stage are dealt to kProducers threads -----
-        const int pid = warp == 0 ? 0 : warp - 9;
-        if (lane == 0) {
-            int stage = 0, round = 0, issued = 0;
-            bool live = true;
-            for (int j = 0; live && j < n_items; ++j) {
-                const int vt = cluster + (j / nG) * n_clusters, tb = 4 * (j % nG);
-                const int v0 = vt * kTileNMax;
-                const int left = h.V - v0;
-                const int N = left >= kTileNMax ? kTileNMax : ((left + 31) / 32) * 32;   // both halves multiples of 16
-                const int half = N >> 1;
-                // bytes of both blocks: every existing M tile of the group + the whole W tile
-                int tiles = 0;
-                for (int q = 0; q < 4; ++q) tiles += (tb + q < nM) ? 1 : 0;
-                const uint32_t bytes = (uint32_t)(tiles * kABytes + N * kTileK * 2);
-                const int my0 = tb + (int)rank, my1 = tb + 2 + (int)rank;           // this block's two M tiles
-                for (int ks = 0; ks < nK; ++ks) {
-                    if (!ptx::mbar_wait(ptx::smem_u32(&s_empty[stage]), (uint32_t)((round & 1) ^ 1), &s_abort)) {
-                        if (!s_abort) raise_abort(&s_abort, t.stat, 0x221u);
-                        live = false;
-                        break;
-                    }
-                    const uint32_t full_local = ptx::smem_u32(&s_full[stage]);
-                    const uint32_t full = ptx::mapa(full_local, 0);                // the leader's barrier
-                    if (rank == 0 && pid == 0) ptx::mbar_arrive_expect_tx(full_local, bytes);
-                    const uint32_t a_dst = ring + (uint32_t)(stage * kStagePBytes);
-                    const uint32_t b_dst = a_dst + 2u * kABytes;
-                    if (my0 < nM && pid == 0)
-                        ptx::tma_g2s_2d_pair(a_dst, &tm_hidden, ks * kTileK, my0 * kTileM, full);
-                    if (my1 < nM && pid == 1 % kProducers)
-                        ptx::tma_g2s_2d_pair(a_dst + kABytes, &tm_hidden, ks * kTileK, my1 * kTileM, full);
-                    int r = 0, op = 2;
-#pragma unroll
-                    for (int b = 3; b >= 0; --b) {
-                        const int rows = 16 << b;
-                        if (half - r >= rows) {
-                            if (op % kProducers == pid)
-                                ptx::tma_g2s_2d_pair(b_dst + (uint32_t)r * 128u, &tm_w.box[b], ks * kTileK,
-                                                     v0 + (int)rank * half + r, full);
-                            r += rows;
-                            ++op;
-                        }
-                    }
-                    ++issued;
-                    if (++stage == kStagesP) { stage = 0; ++round; }
-                }
-            }
-            if (s_abort && rank == 0 && pid == 0) {
-                // no copy may still be landing when the blocks exit; the leader's barriers see both blocks' bytes
-                int first = issued > kStagesP ? issued - kStagesP : 0;
-                for (int q = first; q < issued; ++q)
-                    ptx::mbar_wait(ptx::smem_u32(&s_full[q % kStagesP]), (uint32_t)((q / kStagesP) & 1), &s_zero);
-            }
-        }
-        __syncwarp();
-    } else if (warp == 1) {
-        // ---- MMA issuer (leader only) ---------------------------------------------------------
-        if (lane == 0 && rank == 0) {
-            int stage = 0, round = 0;
-            bool live = true;
-            for (int j = 0; live && j < n_items; ++j) {
-                const int vt = cluster + (j / nG) * n_clusters, tb = 4 * (j % nG);
-                const int left = h.V - vt * kTileNMax;
-                const int N = left >= kTileNMax ? kTileNMax : ((left + 31) / 32) * 32;
-                const bool two = (tb + 2 < nM);
-                if (!ptx::mbar_wait(ptx::smem_u32(&s_acc_empty), (uint32_t)((j & 1) ^ 1), &s_abort)) {
-                    if (!s_abort) raise_abort(&s_abort, t.stat, 0x222u);
-                    break;
-                }
-                ptx::tc_fence_after_sync();
-                const uint32_t idesc = ptx::umma_idesc_bf16(2 * kTileM, N);
-                for (int ks = 0; ks < nK; ++ks) {
-                    if (!ptx::mbar_wait(ptx::smem_u32(&s_full[stage]), (uint32_t)(round & 1), &s_abort)) {
-                        if (!s_abort) raise_abort(&s_abort, t.stat, 0x223u);
-                        live = false;
-                        break;
-                    }
-                    ptx::tc_fence_after_sync();
-                    const uint32_t a_src = ring + (uint32_t)(stage * kStagePBytes);
-                    const uint64_t a0_desc = ptx::smem_desc_sw128(a_src);
-                    const uint64_t a1_desc = ptx::smem_desc_sw128(a_src + kABytes);
-                    const uint64_t b_desc = ptx::smem_desc_sw128(a_src + 2u * kABytes);
-#pragma unroll
-                    for (int kk = 0; kk < kTileK / 16; ++kk)
-                        ptx::umma_bf16_pair(tmem_base, a0_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2),
-                                            idesc, (uint32_t)((ks | kk) != 0));
-                    if (two) {
-#pragma unroll
-                        for (int kk = 0; kk < kTileK / 16; ++kk)
-                            ptx::umma_bf16_pair(tmem_base + kTileNMax, a1_desc + (uint64_t)(kk * 2),
-                                                b_desc + (uint64_t)(kk * 2), idesc, (uint32_t)((ks | kk) != 0));
-                    }
-                    ptx::umma_commit_pair_mcast(ptx::smem_u32(&s_empty[stage]), (uint16_t)3);   // frees the stage in both blocks
-                    if (++stage == kStagesP) { stage = 0; ++round; }
-                }
-                if (live) ptx::umma_commit_pair_mcast(ptx::smem_u32(&s_acc_full), (uint16_t)3);
-            }
-            if (n_items > 0) {
-                ptx::umma_commit_pair(ptx::smem_u32(&s_done));
-                ptx::mbar_wait(ptx::smem_u32(&s_done), 0u, &s_zero);
-            }
-        }
-        __syncwarp();
-    } else {
-        // ---- epilogue (both blocks): warps 2-5 drain the first accumulator, 6-9 the second -----
-        const int acc = (warp - 2) >> 2;
-        const int quarter = warp & 3;
-        const uint32_t acc_empty_leader = ptx::mapa(ptx::smem_u32(&s_acc_empty), 0);
-        for (int j = 0; j < n_items; ++j) {
-            const int vt = cluster + (j / nG) * n_clusters, tb = 4 * (j % nG);
-            const int v0 = vt * kTileNMax;
-            const int left = h.V - v0;
-            const int N = left >= kTileNMax ? kTileNMax : ((left + 31) / 32) * 32;
-            const int tile = tb + 2 * acc + (int)rank;
-            const int row0 = tile * kTileM + quarter * 32;
-            const int row = row0 + lane;
-            if (!ptx::mbar_wait(ptx::smem_u32(&s_acc_full), (uint32_t)(j & 1), &s_abort)) {
-                if (lane == 0 && !s_abort) raise_abort(&s_abort, t.stat, 0x224u);
-                break;
-            }
-            ptx::tc_fence_after_sync();
-            Stats st = stats_empty();
-            const bool warp_has_rows = tile < nM && row0 < R_live;
-            if (warp_has_rows) {
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kTileNMax);
-                for (int c0 = 0; c0 < N; c0 += 32) {
-                    float z[32];
-                    ptx::tmem_ld_32x32(taddr + (uint32_t)c0, z);
-                    int n_valid = N - c0;
-                    if (h.V - (v0 + c0) < n_valid) n_valid = h.V - (v0 + c0);
-                    if (n_valid > 32) n_valid = 32;
-                    if (row < R_live && n_valid > 0) fold_chunk(st, z, n_valid, v0 + c0, h.sample, (uint32_t)row);
-                }
-            }
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(acc_empty_leader);
-            if (warp_has_rows && row < R_live)
-                partial_store(P, (size_t)row * n_slices + (size_t)vt, st);
-        }
-    }
-
-    ptx::tc_fence_before_sync();
-    __threadfence();
-    __syncthreads();
-    ptx::cluster_sync();               // neither block leaves while the pair may still touch its memory
-    if (warp == 1) {
-        ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
-    }
-}
-
 // hidden[row_idx[r]] -> packed[r] (zero for rows past the live count or with a bad index).
 __global__ void __launch_bounds__(128)
 gather_rows_kernel(HeadArgs h, uint4 *packed, int rows_padded, DevStat *stat)
@@ -1021,7 +802,7 @@ size_t umma_gather_bytes(int R, int d)
 static_assert(sizeof(CUtensorMap) == sizeof(TmapCache::Entry::map), "tensor-map cache entry size");
 
 cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch &s, void *gather_buf,
-                             int sm_count, cudaStream_t stream, int *launched, bool use_pair, TmapCache *cache)
+                             int sm_count, cudaStream_t stream, int *launched, TmapCache *cache)
 {
     *launched = 0;
     static bool configured[64] = {};
@@ -1032,8 +813,6 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
         e = cudaFuncSetAttribute(head_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmem);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(head_umma2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmem2);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(head_umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemP);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -1087,18 +866,6 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
     if (plan.nM == 1) {
         void *args[] = {&tm_h, &tm_w, &hk2, &tk, &Pk, &plan};
         e = launch_dependent((const void *)head_umma_kernel, dim3((unsigned)grid), dim3(kThreads), kDynSmem, stream, args);
-    } else if (use_pair && grid >= 2) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(grid & ~1));
-        cfg.blockDim = dim3(kThreadsP);
-        cfg.dynamicSmemBytes = kDynSmemP;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, head_umma_pair_kernel, tm_h, tm_w, hk, t, P, plan.nM, plan.n_slices);
     } else {
         void *args[] = {&tm_h, &tm_w, &hk2, &tk, &Pk, &plan.nM, &plan.n_slices};
         e = launch_dependent((const void *)head_umma2_kernel, dim3((unsigned)grid), dim3(kThreads2), kDynSmem2, stream, args);

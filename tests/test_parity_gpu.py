@@ -85,13 +85,6 @@ def test_tensor_core_path_shapes(rs, handle, oracle, B, d, V):
     check_case(rs, handle, oracle, w, [0, 1], flags=rs.PATH_UMMA)
 
 
-@pytest.mark.parametrize("B,d,V", [(129, 64, 777), (300, 256, 4099), (544, 320, 1031)])
-def test_tensor_core_block_pair_variant_for_many_rows(rs, handle, oracle, B, d, V):
-    # more than 128 rows on pairs of blocks (cta_group::2): four M tiles per W tile and pair
-    w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=d, V=V, seed=9100 + B + d + V, sigma_w=0.5 / math.sqrt(d))
-    check_case(rs, handle, oracle, w, [0], flags=rs.PATH_UMMA | rs.PATH_PAIR)
-
-
 def test_tensor_core_path_gather_live_count_and_spans(rs, handle, oracle):
     # row gather + device-side live row count, then multi-row spans over several M tiles
     w = gen.scaled(gen.WORKLOADS["c4_llm_b64"], V=3000, d=512, B=64)
