@@ -505,3 +505,43 @@ def test_random_shapes_sweep(rs, handle, oracle):
         except AssertionError as e:
             raise AssertionError("case %d: B=%d d=%d V=%d path=%s: %s" % (done, B, d, V, path, e))
         done += 1
+
+
+def test_back_to_back_calls_share_one_scratch(rs, handle, oracle):
+    # A call's head kernel is allowed to start while the call before it on the stream is still merging
+    # its partial statistics (programmatic dependent launch); the two share the handle's scratch.  A long
+    # train of calls of mixed shapes, row counts and kernel families is enqueued without any host
+    # synchronisation, every call into its own output buffers, the inputs of call i + 1 written by a
+    # copy kernel enqueued right behind call i; afterwards every call's decision is compared with the
+    # oracle's.  A head kernel that read its hidden rows, or wrote the scratch, before the kernels ahead
+    # of it had finished would show up here.
+    import torch
+    shapes = [(1, 512, 9001), (16, 256, 4099), (1, 64, 300), (64, 320, 5003), (3, 128, 2000), (130, 256, 2304),
+              (2, 1024, 30011), (40, 64, 777)]
+    cases = []
+    for k, (B, d, V) in enumerate(shapes):
+        w = gen.scaled(gen.WORKLOADS["c4_slm_b64"], B=B, d=d, V=V, seed=9700 + k, sigma_w=0.5 / math.sqrt(d))
+        w_bits = gen.make_w_head(w)
+        hids = [gen.make_hidden(w, w_bits, s)[0] for s in range(3)]
+        cases.append({"w": w, "w_bits": w_bits, "w_dev": to_dev_bf16(w_bits), "hid_bits": hids,
+                      "staged": [to_dev_bf16(h) for h in hids],                 # where the inputs wait
+                      "live": torch.zeros((B, d), dtype=torch.bfloat16, device="cuda")})   # what the calls read
+    order = [(k, s) for s in range(3) for k in range(len(cases))]
+    outs = [rs.RouteOutputs.allocate(cases[k]["w"].B, cases[k]["w"].B, "cuda") for k, _ in order]   # (fills: kernels)
+    torch.cuda.synchronize()
+    for (k, s), out in zip(order, outs):
+        c = cases[k]
+        if s == 1:
+            hid = c["staged"][s]                         # nothing between this call and the one before it
+        else:
+            hid = c["live"]
+            hid.copy_(c["staged"][s])                    # a kernel right in front of the call writes its input
+        rs.route_ex(handle, hid, c["w_dev"], c["w"].tau_nats, out=out)
+    torch.cuda.synchronize()
+    for (k, s), out in zip(order, outs):
+        c = cases[k]
+        w = c["w"]
+        gpu = {n: getattr(out, n).cpu().numpy() for n in ("tok", "ent", "mask", "llm_idx", "llm_count")}
+        compare(gpu, oracle.route(c["hid_bits"][s], c["w_bits"], w.tau_nats), w.tau_nats, w.B, w.B)
+    st = rs.last_status(handle)
+    assert st["timeouts"] == 0 and st["nan_rows"] == 0
