@@ -30,6 +30,16 @@
  *  - Calls are asynchronous on the given CUDA stream: outputs are valid once
  *    that stream has been synchronised.  llm_count stays on the device so that
  *    the next model's step can be enqueued without a host round trip.
+ *  - Host threads: a handle, and the per-device internal handle behind the entry points that take none
+ *    (rstitch_route, rstitch_compact, rstitch_route_static's set-up), may be used by one host thread at
+ *    a time.  Different handles may be used from different threads at once.
+ *  - A routing call enqueues two kernels (the head kernel and the kernel that merges its per-block
+ *    statistics and decides) with programmatic stream serialisation: the call's own head kernel may begin
+ *    to read W_head while the kernel before it on the stream is still running, and waits for that kernel
+ *    to complete before it reads anything else.  W_head must therefore not be written by a kernel
+ *    that may still be running then -- the kernel enqueued directly before the call on the same stream
+ *    and, if that one was itself launched with programmatic serialisation, those before it (weights are
+ *    not expected to be); every other input may be.
  *  - bf16 tensors are row-major with the contraction index k contiguous.
  *  - Non-finite inputs: a row whose entropy is NaN is routed (mask = 1), its
  *    token is the lowest index of the largest non-NaN logit (0 if none), and
@@ -193,7 +203,9 @@ int rstitch_route_ex_host(rstitch_handle_t h, const rstitch_args_t *a, void *cud
  *  - All calls on a device share the one array, which keeps the previous call's contents: each call
  *    clears what must start at zero on the given stream.  Two calls that overlap on the GPU (different
  *    streams, no ordering between them) race on it; order them.
- *  - No status word is reported back: NaN rows are still routed, but not counted anywhere.
+ *  - No status word is reported back: NaN rows are still routed, but not counted anywhere, and a bounded
+ *    device-side wait that gave up (which the other entry points report through rstitch_last_status as
+ *    RSTITCH_ERR_TIMEOUT) goes unreported here; the outputs of such a call are undefined.
  */
 #define RSTITCH_STATIC_MAX_ROWS 16
 int rstitch_route_static(const void *hidden /* bf16 [B,d] */, const void *W_head /* bf16 [V,d] */,

@@ -35,12 +35,12 @@ head_finalize_kernel(Partials P, int n_slices, int R, const int32_t *n_rows_dev,
     if (n_rows_dev) { int n = *n_rows_dev; R_live = n < 0 ? 0 : (n < R ? n : R); }
     const int lane = threadIdx.x & 31;
     for (int r = blockIdx.x * kFinRows + (threadIdx.x >> 5); r < R_live; r += gridDim.x * kFinRows) {
-        Stats st;
-        if (n_slices <= 256) {
-            st = tail_row_direct(P, (size_t)r * n_slices, n_slices, lane);
-        } else {
-            st = tail_merge_strided(P, (size_t)r * n_slices, n_slices, lane, 32);
-            stats_warp_allmerge(st);
+        // 256 slices at a time: one round trip to L2 per chunk with every load in flight, chunks merged in
+        // ascending order (the many-row kernel leaves one partial per 256-row vocabulary tile: 594 of them)
+        Stats st = tail_row_direct(P, (size_t)r * n_slices, n_slices < 256 ? n_slices : 256, lane);
+        for (int c0 = 256; c0 < n_slices; c0 += 256) {
+            const Stats more = tail_row_direct(P, (size_t)r * n_slices + c0, n_slices - c0 < 256 ? n_slices - c0 : 256, lane);
+            stats_merge(st, more);
         }
         if (lane == 0) {
             const float H = tail_emit_row(st, r, t);

@@ -80,25 +80,4 @@ __device__ __forceinline__ void stats_merge(Stats &a, const Stats &b)
     a.m = M; a.s = s; a.u = u;
 }
 
-__device__ __forceinline__ Stats stats_shfl_xor(const Stats &t, int lane_mask)
-{
-    Stats o;
-    o.m  = __shfl_xor_sync(0xffffffffu, t.m, lane_mask);
-    o.s  = __shfl_xor_sync(0xffffffffu, t.s, lane_mask);
-    o.u  = __shfl_xor_sync(0xffffffffu, t.u, lane_mask);
-    o.bv = __shfl_xor_sync(0xffffffffu, t.bv, lane_mask);
-    o.bi = __shfl_xor_sync(0xffffffffu, t.bi, lane_mask);
-    return o;
-}
-
-// All lanes end with the merge of the 32 lanes' sets, in a fixed butterfly order.
-__device__ __forceinline__ void stats_warp_allmerge(Stats &t)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        Stats p = stats_shfl_xor(t, o);
-        stats_merge(t, p);
-    }
-}
-
 }  // namespace rstitch

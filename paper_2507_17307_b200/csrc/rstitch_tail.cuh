@@ -99,29 +99,6 @@ __device__ __forceinline__ float tail_emit_row(const Stats &t, int r, const Tail
     return H;
 }
 
-// Merge of slices part, part + parts, ... of one row by one thread, loads issued four at a time.
-__device__ __forceinline__ Stats tail_merge_strided(const Partials &P, size_t row_base, int n_slices,
-                                                    int part, int parts)
-{
-    Stats t = stats_empty();
-    int c = part;
-    for (; c + 3 * parts < n_slices; c += 4 * parts) {
-        Stats p0 = partial_load(P, row_base + c);
-        Stats p1 = partial_load(P, row_base + c + parts);
-        Stats p2 = partial_load(P, row_base + c + 2 * parts);
-        Stats p3 = partial_load(P, row_base + c + 3 * parts);
-        stats_merge(p0, p1);
-        stats_merge(p2, p3);
-        stats_merge(p0, p2);
-        stats_merge(t, p0);
-    }
-    for (; c < n_slices; c += parts) {
-        Stats p = partial_load(P, row_base + c);
-        stats_merge(t, p);
-    }
-    return t;
-}
-
 // One row's n_slices <= 256 partials merged by one warp: every partial of the row is pulled into
 // registers with all loads in flight at once (a single round trip to L2), then merged without a
 // dependent chain: the row maximum M and the greedy token first, then one exponential per partial for
