@@ -214,15 +214,19 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ring = (ptx::smem_u32(dyn_smem_raw) + 1023u) & ~1023u;
     const int nK = (h.d + kTileK - 1) / kTileK;
-    int R_live = h.R;
-    // A live row count on the device is the output of an earlier kernel: wait for it.  Without one the
-    // producer starts on W_head (a weight no earlier kernel writes) at once and waits only before its
-    // first copy of hidden rows.
-    if (h.n_rows_dev) { ptx::grid_dep_wait(); int n = *h.n_rows_dev; R_live = n < 0 ? 0 : (n < h.R ? n : h.R); }
+    // The live row count, when it sits on the device, is the output of an earlier kernel, and so may the
+    // hidden rows be; W_head is not.  Every role therefore waits for the kernels before this one by itself,
+    // as late as it can: the producer only after a first ring of W_head has been asked for, the others
+    // when they first need the count.
+    auto rows_live = [&]() -> int {
+        if (!h.n_rows_dev) return h.R;
+        ptx::grid_dep_wait();
+        const int n = *h.n_rows_dev;
+        return n < 0 ? 0 : (n < h.R ? n : h.R);
+    };
 
     Schedule sch;
     sch.init(h.V, gridDim.x, blockIdx.x, plan.tiles_per_block);
-    if (R_live == 0) sch.n_items = 0;          // no live rows (device-side count): nothing to stream
 
     if (threadIdx.x == 0) {
         s_abort = 0; s_zero = 0;
@@ -258,7 +262,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
             // pass over the ring is complete only the W parts of the stages are fetched, and the hidden
             // tiles owed to those stages are remembered; then the producer waits for the earlier kernels,
             // pays the debt and goes on with whole stages.  A ring of W_head is in flight meanwhile.
-            bool waited = (h.n_rows_dev != nullptr);
+            bool waited = false, no_rows = false;
             uint32_t owed_full[kMaxStages], owed_dst[kMaxStages];
             int owed_x[kMaxStages], n_owed = 0;
             auto settle = [&]() {
@@ -266,6 +270,9 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                 for (int q = 0; q < n_owed; ++q) ptx::tma_g2s_2d(owed_dst[q], &tm_hidden, owed_x[q], 0, owed_full[q]);
                 n_owed = 0;
                 waited = true;
+                // no live row after all (a count on the device): the stages asked for so far complete, nobody
+                // consumes them, and the producer only sees them land before it leaves
+                if (h.n_rows_dev && *h.n_rows_dev <= 0) { no_rows = true; live = false; }
             };
             for (int j = 0; live && j < sch.n_items; ++j) {
                 const Item it = sch.item(j);
@@ -277,6 +284,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                     int ng = nK - ks < kIssueGroup ? nK - ks : kIssueGroup;
                     if (ng > n_stages) ng = n_stages;
                     if (!waited && issued + ng > n_stages) settle();     // the ring has been round once
+                    if (!live) break;
                     uint32_t full[kIssueGroup], a_dst[kIssueGroup];
                     for (int g = 0; g < ng; ++g) {
                         int sg = stage + g, rd = round;
@@ -319,7 +327,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
                 }
             }
             if (!waited) settle();                   // fewer k-steps than stages: every armed stage gets its hidden tile
-            if (s_abort && pid == 0) {
+            if ((s_abort || no_rows) && pid == 0) {
                 // no copy may still be landing in this block's shared memory when it exits
                 int first = issued > n_stages ? issued - n_stages : 0;
                 for (int q = first; q < issued; ++q)
@@ -332,6 +340,7 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
         if (lane == 0) {
             int stage = 0, round = 0;
             bool live = true;
+            if (rows_live() == 0) sch.n_items = 0;       // no live rows (device-side count): nothing to multiply
             for (int j = 0; live && j < sch.n_items; ++j) {
                 const Item it = sch.item(j);
                 const int buf = j & 1, use = j >> 1;
@@ -375,6 +384,8 @@ head_umma_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_con
         // ---- epilogue: warps 2-5 fold the first half of a tile's 32-column chunks, warps 6-9 the rest ----
         const int quarter = warp & 3;                        // the TMEM lanes this warp may read
         const int half = (warp - 2) >> 2;
+        const int R_live = rows_live();
+        if (R_live == 0) sch.n_items = 0;
         // M = 128: accumulator row i is lane i.  M = 64: row i is lane 32 (i / 16) + i % 16.
         const int rows_per_quarter = plan.m64 ? 16 : 32;
         const int row = quarter * rows_per_quarter + lane;
@@ -709,6 +720,10 @@ head_umma2_kernel(const __grid_constant__ CUtensorMap tm_hidden, const __grid_co
 __global__ void __launch_bounds__(128)
 gather_rows_kernel(HeadArgs h, uint4 *packed, int rows_padded, DevStat *stat)
 {
+    // the head kernel behind this one may start on W_head at once; it waits for this kernel before it
+    // reads the packed rows, as this kernel waits for the ones that wrote the index list and the count
+    ptx::grid_dep_launch_dependents();
+    ptx::grid_dep_wait();
     const int r = blockIdx.x;
     const int d8 = h.d >> 3;
     int R_live = h.R;
@@ -847,8 +862,12 @@ cudaError_t launch_head_umma(const HeadArgs &h, const TailArgs &t, const Scratch
     if (h.row_idx) {
         // the tensor-map copy cannot follow an index list: pack the gathered rows first
         const int rows_padded = plan.nM * kTileM;
-        gather_rows_kernel<<<rows_padded, 128, 0, stream>>>(h, (uint4 *)gather_buf, rows_padded, t.stat);
-        e = cudaGetLastError();
+        HeadArgs hg = h;
+        uint4 *packed = (uint4 *)gather_buf;
+        int padded = rows_padded;
+        DevStat *stat = t.stat;
+        void *gargs[] = {&hg, &packed, &padded, &stat};
+        e = launch_dependent((const void *)gather_rows_kernel, dim3((unsigned)rows_padded), dim3(128), 0, stream, gargs);
         if (e != cudaSuccess) return e;
         ++*launched;
         hid_base = gather_buf;
