@@ -132,19 +132,25 @@ def measured_peaks() -> dict:
             "bf16_tflops_sustained": FALLBACK_BF16_TFLOPS_SUSTAINED, "source": "fallback"}
 
 
-# DRAM bytes (read + write) per launch of the dominant kernel, from the ncu captures summarised under
+# DRAM bytes (read + write) per launch of the dominant (head) kernel, from the ncu captures summarised under
 # profiles/.  Each entry names the kernel sources it was taken with (sha256 of the files under csrc/):
 # once any of them has changed the counters no longer describe the kernel and the figure reads null.
 NCU_TRAFFIC = {
     "c2_slm_b1":
-    {"bytes": 471337088, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
-     "sources": {"rstitch_gemv.cu": "6cb7364043bc168af40c7326f453cbad357801df952106ad47c0eb9a454bae6c", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "cd4da5f27447a88d28393e5aa40a8d6bdecfbe7ab8da0e06d678a01268d9b48f", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 470788736, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
+     "sources": {"rstitch_gemv.cu": "46622a9ca185e4b62ecd29c125a00875a0d28e9416790789c855643721c5222e", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
+    "c3_llm_b1":
+    {"bytes": 1094061028, "summary": "profiles/head_stream_kernel_c3_llm_b1.md",
+     "sources": {"rstitch_gemv.cu": "46622a9ca185e4b62ecd29c125a00875a0d28e9416790789c855643721c5222e", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
+    "c3_llm_b16":
+    {"bytes": 1095153244, "summary": "profiles/head_umma_kernel_c3_llm_b16.md",
+     "sources": {"rstitch_umma.cu": "71930ba3f0ec83a8479520e7eea7171908ed223a08bfbf93968346a06c57164f", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
     "c4_slm_b64":
-    {"bytes": 472086784, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
-     "sources": {"rstitch_umma.cu": "b0f379310c237b685275d916050df3d5b03d32f0860c865a399007a73dba3a39", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "cd4da5f27447a88d28393e5aa40a8d6bdecfbe7ab8da0e06d678a01268d9b48f", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 471473664, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
+     "sources": {"rstitch_umma.cu": "71930ba3f0ec83a8479520e7eea7171908ed223a08bfbf93968346a06c57164f", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
     "c5_catchup":
-    {"bytes": 1667069088, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
-     "sources": {"rstitch_umma.cu": "b0f379310c237b685275d916050df3d5b03d32f0860c865a399007a73dba3a39", "rstitch_kernels.cuh": "700af071b27232beeee2b60b10c2442e0c6ed50d424e5522af1818a80f707f79", "rstitch_tail.cuh": "cd4da5f27447a88d28393e5aa40a8d6bdecfbe7ab8da0e06d678a01268d9b48f", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "49a7c5499dcb8af16e566d75ff13f95b18899a5c1fa38c9947a31c43763b1769", "rstitch_ptx.cuh": "f52963337289b5daf617e154b5b5e403e0a22a92f1a4502864243a86e967200e", "rstitch_sample.cuh": "d21659a3db5bc1f95b560f0ae71c4a71c063816d1e5aa85e4ee58acf044ce1a2"}},
+    {"bytes": 1675168104, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
+     "sources": {"rstitch_umma.cu": "71930ba3f0ec83a8479520e7eea7171908ed223a08bfbf93968346a06c57164f", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
 }
 
 
