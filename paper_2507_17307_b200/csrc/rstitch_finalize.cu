@@ -48,15 +48,10 @@ head_finalize_kernel(Partials P, int n_slices, int R, const int32_t *n_rows_dev,
         }
     }
     if (gridDim.x > 1) {
-        __threadfence();
+        __syncthreads();             // the block's rows are written ...
+        if (threadIdx.x == 0) s_last = (ptx::ticket_take(ticket) == gridDim.x - 1);   // ... and released with its ticket
         __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned k = atomicAdd(ticket, 1u);
-            s_last = (k == gridDim.x - 1);
-        }
-        __syncthreads();
-        if (!s_last) return;
-        __threadfence();
+        if (!s_last) return;         // the last ticket has acquired every other block's rows
     } else {
         __syncthreads();
     }

@@ -98,6 +98,17 @@ __device__ __forceinline__ void grid_dep_wait()
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// ---- tickets -------------------------------------------------------------------------------
+// One block's ticket from a counter in global memory as a single acquire-release operation at GPU scope:
+// what the block's threads stored before the barrier in front of this call is visible to whoever draws a
+// later ticket, without a separate fence and its round trip on either side.
+__device__ __forceinline__ unsigned ticket_take(unsigned *counter)
+{
+    unsigned k;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(k) : "l"(counter) : "memory");
+    return k;
+}
+
 // ---- bulk copies ------------------------------------------------------------------------
 // Untiled copy global -> shared; both addresses 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
