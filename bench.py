@@ -137,20 +137,20 @@ def measured_peaks() -> dict:
 # once any of them has changed the counters no longer describe the kernel and the figure reads null.
 NCU_TRAFFIC = {
     "c2_slm_b1":
-    {"bytes": 470788736, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
-     "sources": {"rstitch_gemv.cu": "46622a9ca185e4b62ecd29c125a00875a0d28e9416790789c855643721c5222e", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
+    {"bytes": 470766592, "summary": "profiles/head_stream_kernel_c2_slm_b1.md",
+     "sources": {"rstitch_gemv.cu": "46622a9ca185e4b62ecd29c125a00875a0d28e9416790789c855643721c5222e", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "3b15b917fd957debc456aa9fe0e557fa4769f476479b08233d396504eb3cdf8c", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "7c388069cec80e69781d2fc0a46b5d6a71aeed12db1bc249e0bc60adb9f80107"}},
     "c3_llm_b1":
-    {"bytes": 1094061028, "summary": "profiles/head_stream_kernel_c3_llm_b1.md",
-     "sources": {"rstitch_gemv.cu": "46622a9ca185e4b62ecd29c125a00875a0d28e9416790789c855643721c5222e", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
+    {"bytes": 1094197912, "summary": "profiles/head_stream_kernel_c3_llm_b1.md",
+     "sources": {"rstitch_gemv.cu": "46622a9ca185e4b62ecd29c125a00875a0d28e9416790789c855643721c5222e", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "3b15b917fd957debc456aa9fe0e557fa4769f476479b08233d396504eb3cdf8c", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "7c388069cec80e69781d2fc0a46b5d6a71aeed12db1bc249e0bc60adb9f80107"}},
     "c3_llm_b16":
-    {"bytes": 1095153244, "summary": "profiles/head_umma_kernel_c3_llm_b16.md",
-     "sources": {"rstitch_umma.cu": "71930ba3f0ec83a8479520e7eea7171908ed223a08bfbf93968346a06c57164f", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
+    {"bytes": 1094429312, "summary": "profiles/head_umma_kernel_c3_llm_b16.md",
+     "sources": {"rstitch_umma.cu": "71930ba3f0ec83a8479520e7eea7171908ed223a08bfbf93968346a06c57164f", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "3b15b917fd957debc456aa9fe0e557fa4769f476479b08233d396504eb3cdf8c", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "7c388069cec80e69781d2fc0a46b5d6a71aeed12db1bc249e0bc60adb9f80107"}},
     "c4_slm_b64":
-    {"bytes": 471473664, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
-     "sources": {"rstitch_umma.cu": "71930ba3f0ec83a8479520e7eea7171908ed223a08bfbf93968346a06c57164f", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
+    {"bytes": 471256832, "summary": "profiles/head_umma_kernel_c4_slm_b64.md",
+     "sources": {"rstitch_umma.cu": "71930ba3f0ec83a8479520e7eea7171908ed223a08bfbf93968346a06c57164f", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "3b15b917fd957debc456aa9fe0e557fa4769f476479b08233d396504eb3cdf8c", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "7c388069cec80e69781d2fc0a46b5d6a71aeed12db1bc249e0bc60adb9f80107"}},
     "c5_catchup":
-    {"bytes": 1675168104, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
-     "sources": {"rstitch_umma.cu": "71930ba3f0ec83a8479520e7eea7171908ed223a08bfbf93968346a06c57164f", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "0e62a2c6a6b306c74395d61dd31dd18283ca386b7b71d37a28e559e51e08b908", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "3046b6fb0ba11d03ceaa0c0c171b310a8f14ae0e5f9d58fff6ac18fdf457ff85"}},
+    {"bytes": 1673064760, "summary": "profiles/head_umma2_kernel_c5_catchup.md",
+     "sources": {"rstitch_umma.cu": "71930ba3f0ec83a8479520e7eea7171908ed223a08bfbf93968346a06c57164f", "rstitch_kernels.cuh": "9d5e477d91dc22a265a8430f1ac19aba750e147118779e27533337225eba6f34", "rstitch_tail.cuh": "6f57211cd838c59082c6ae636fc198557d5a6c8a6a4bda2d4a48324bb8541ce6", "rstitch_alg1.cuh": "a14e9fd9944096aff664d96854f70a356e706967772dc0d918a7f7fcccc55f0f", "rstitch_stats.cuh": "e9ff9c67605d61e89d9db77ba12376630bd3a612160977946ac7e2aadd51542e", "rstitch_ptx.cuh": "3b15b917fd957debc456aa9fe0e557fa4769f476479b08233d396504eb3cdf8c", "rstitch_sample.cuh": "40e02e3cd65cde7d19108dd6ae55f59fc1d1b0ee1171efe6f0de23e5cff04f71", "rstitch_finalize.cu": "7c388069cec80e69781d2fc0a46b5d6a71aeed12db1bc249e0bc60adb9f80107"}},
 }
 
 
