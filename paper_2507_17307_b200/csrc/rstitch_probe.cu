@@ -70,9 +70,10 @@ read_stream_kernel(const unsigned char *src, unsigned long long n_chunks, unsign
 extern "C" int rstitch_probe_read_stream(const void *buf, size_t bytes, uint32_t *gave_up, void *cuda_stream)
 {
     using namespace rstitch;
-    if (!buf || !gave_up || (reinterpret_cast<uintptr_t>(buf) % 16) != 0) return RSTITCH_ERR_INVALID_ARG;
+    if (!gave_up) return RSTITCH_ERR_INVALID_ARG;
     const unsigned long long n_chunks = bytes / kProbeChunk;
-    if (n_chunks == 0) return RSTITCH_OK;
+    if (n_chunks == 0) return RSTITCH_OK;                 // less than one chunk: nothing is read
+    if (!buf || (reinterpret_cast<uintptr_t>(buf) % 16) != 0) return RSTITCH_ERR_INVALID_ARG;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1 ||

@@ -107,3 +107,40 @@ def test_router_argument_errors(rs):
     big = rs.Router(dev_weights(gen.make_router_weights(64, 300, 16, 1, seed=1)))
     assert big.forward(hid, 4, check=False) == -3
     assert r.forward(hid, 0)[0] is not None                                  # empty batch is fine
+
+
+def test_router_bad_index_decides_nothing(rs, oracle):
+    # an entry of row_idx outside [0, n_src) reads row 0, gets switch 0 and leaves the mask alone
+    # (it used to refine sequence 0's decision); rows to read with no row present is an argument error
+    import torch
+    d, n_src = 128, 6
+    w = gen.make_router_weights(d, 16, 32, 2, seed=3)
+    router = rs.Router(dev_weights(w))
+    hid_bits = gen.f32_to_bf16_bits((np.random.default_rng(1).standard_normal((n_src, d)) * 2.0).astype(np.float32))
+    hid = to_dev_bf16(hid_bits)
+    idx = np.array([4, -1, 2, 99, 0], dtype=np.int32)
+    mask = torch.full((n_src,), 7, dtype=torch.uint8, device="cuda")
+    logits, sw = router.forward(hid, idx.size, row_idx=to_dev_i32(idx), refine_mask=mask)
+    torch.cuda.synchronize()
+    ref_logits, ref_sw = oracle.router_rows(hid_bits, w, row_idx=np.array([4, 0, 2, 0, 0], dtype=np.int32))
+    got_sw, got_mask = sw.cpu().numpy()[:idx.size], mask.cpu().numpy()
+    assert np.abs(logits.cpu().numpy()[:idx.size] - ref_logits).max() <= LOGIT_TOL
+    good = np.array([0, 2, 4])
+    assert np.array_equal(got_sw[good], ref_sw[good]) and (got_sw[[1, 3]] == 0).all()
+    assert got_mask[4] == ref_sw[0] and got_mask[2] == ref_sw[2] and got_mask[0] == ref_sw[4]
+    assert (got_mask[[1, 3, 5]] == 7).all()                      # untouched
+    empty = torch.zeros((0, d), dtype=torch.bfloat16, device="cuda")
+    assert router.forward(empty, 2, row_idx=to_dev_i32([0, 0]), check=False) == -1
+    torch.cuda.synchronize()
+
+
+def test_read_stream_probe(rs):
+    # the measurement aid: whole 16 KiB chunks are read, nothing is written, no bounded wait runs out
+    import torch
+    gave_up = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for n in (0, 100, 16 * 1024, 5 * 16 * 1024 + 7, 64 << 20):
+        buf = torch.full((n,), 3, dtype=torch.uint8, device="cuda")
+        assert rs.probe_read_stream(buf, gave_up) == 0
+        torch.cuda.synchronize()
+        assert int(gave_up.item()) == 0
+        assert n == 0 or (int(buf[0].item()) == 3 and int(buf[-1].item()) == 3)
