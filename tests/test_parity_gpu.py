@@ -545,3 +545,28 @@ def test_back_to_back_calls_share_one_scratch(rs, handle, oracle):
         compare(gpu, oracle.route(c["hid_bits"][s], c["w_bits"], w.tau_nats), w.tau_nats, w.B, w.B)
     st = rs.last_status(handle)
     assert st["timeouts"] == 0 and st["nan_rows"] == 0
+
+
+@pytest.mark.parametrize("path", ["gemv", "umma"])
+@pytest.mark.parametrize("gather", [False, True])
+def test_live_row_count_of_zero_on_the_device(rs, handle, oracle, path, gather):
+    # a device-side row count of zero (the LLM's batch in a round in which no sequence sits on the LLM): the
+    # head kernel has already asked for its first ring of W_head when it learns that; nothing may be written
+    # but llm_count = 0, no wait may run out, and the very next call on the handle must be a normal one
+    flags = rs.PATH_GEMV if path == "gemv" else rs.PATH_UMMA
+    w = gen.scaled(gen.WORKLOADS["c4_llm_b64"], V=5003, d=512, B=40)
+    w_bits = gen.make_w_head(w)
+    w_dev = to_dev_bf16(w_bits)
+    hid, _ = gen.make_hidden(w, w_bits, 0)
+    row_idx = np.arange(w.B, dtype=np.int32)[::-1].copy() if gather else None
+    for _ in range(3):
+        gpu = run_gpu(handle, hid, w_dev, w.tau_nats, row_idx=row_idx, n_rows_dev=0, R=w.B, flags=flags)
+        assert int(gpu["llm_count"][0]) == 0
+        assert (gpu["tok"] == -1).all() and (gpu["ent"] == -1.0).all()
+        assert (gpu["mask"] == 255).all() and (gpu["llm_idx"] == -1).all()
+    st = rs.last_status(handle)
+    assert st["timeouts"] == 0 and st["nan_rows"] == 0 and st["bad_row_idx"] == 0
+    ref = oracle.route(hid, w_bits, w.tau_nats, row_idx=row_idx)
+    gpu = run_gpu(handle, hid, w_dev, w.tau_nats, row_idx=row_idx, flags=flags)
+    compare(gpu, ref, w.tau_nats, w.B, w.B)
+    assert rs.last_status(handle)["timeouts"] == 0
